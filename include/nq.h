@@ -1,0 +1,197 @@
+/*
+ * nq.h -- C boundary of the B200 (sm_100a) NestQuant hot path.
+ *
+ * NestQuant ("Post-Training Integer-Nesting Quantization for On-Device DNN") stores an INTn
+ * quantised weight as two integers, w_int = w_high * 2^l + w_low with n = h + l (Eq. 5), so that a
+ * model can run "part-bit" on w_high alone (scale inflated to s * 2^l, Eq. 9) and be upgraded to
+ * the "full-bit" INTn model by paging w_low back in and recomposing.  This library is the
+ * data-parallel part of that: decomposition, recomposition, dropping the low part, and the integer
+ * GEMM / convolution on the nested weights in both modes.
+ *
+ * General rules for every entry point
+ *   - Pointers marked (device) are device memory of the current CUDA device, owned by the caller and
+ *     alive until the work queued on `stream` has finished.  Pointers marked (host) are read before
+ *     the call returns.  The library allocates no device memory.
+ *   - `stream` is a cudaStream_t passed as void* (0 = the default stream).  Calls only enqueue work
+ *     and return; they never synchronise, except nq_device_status.
+ *   - Return value: NQ_OK or an nq_status error.  Argument errors are found before anything is
+ *     launched.  Nothing aborts, traps or throws.
+ *   - Weight matrices are [rows, cols] = [output channels, K] with K contiguous.
+ *   - Nesting parameters: n_bits in [2, 8]; h_bits in [1, n_bits - 1]; l = n_bits - h_bits;
+ *     compensate != 0 keeps w_low in l + 1 bits ("Full-Bit Model: Performance Compensation"),
+ *     compensate == 0 clips it to l bits (Eq. 10).  Unpacked weights are int8 holding INTn values;
+ *     for n_bits < 8 values outside [-2^(n-1), 2^(n-1) - 1] give unspecified results.
+ *
+ * Packed ("sliced") layout of a [rows, cols] tensor of k-bit two's-complement fields
+ *   Each row is padded with zero fields to a multiple of 128 and cut into groups of 128 elements;
+ *   a group is 16*k bytes, a row nq_packed_row_bytes(cols, k) bytes, rows follow one another.
+ *   k is split into powers of two (8, 4, 2, 1), widest first; the slice of width s holds s bits of
+ *   every field (the widest slice the most significant bits) in 16*s bytes.  In a slice, element e
+ *   of the group lives in byte ((e/32)*s + ((e%32)/4) / (8/s)) * 4 + e%4, at bits
+ *   [8 - s*(sub+1), 8 - s*sub) with sub = ((e%32)/4) % (8/s).  (The paper only fixes the field
+ *   width and its two's-complement content; this placement lets four fields be extracted with one
+ *   mask per 32-bit word.)  The base address of a packed tensor must be 16-byte aligned.
+ */
+#ifndef NQ_H_
+#define NQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define NQ_API __attribute__((visibility("default")))
+#else
+#define NQ_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    NQ_OK = 0,
+    NQ_ERR_INVALID_ARG = 1, /* null pointer, negative size, inconsistent shapes                 */
+    NQ_ERR_UNSUPPORTED = 2, /* nesting (n, h) or shape outside what the kernels implement        */
+    NQ_ERR_ALIGNMENT = 3,   /* a pointer or pitch breaks the stated alignment rule               */
+    NQ_ERR_WORKSPACE = 4,   /* workspace missing or too small                                    */
+    NQ_ERR_CUDA = 5,        /* a CUDA runtime / driver call failed (launch, descriptor encoding) */
+    NQ_ERR_TIMEOUT = 6      /* a bounded on-device wait expired (reported by nq_device_status)   */
+} nq_status;
+
+typedef enum { NQ_F32 = 0, NQ_BF16 = 1 } nq_dtype;
+
+/* Text for a status code (host, static storage). */
+NQ_API const char *nq_status_str(int status);
+
+/* Bits of the stored low field: l + 1 with compensation, l without.  Returns -1 for a bad (n, h). */
+NQ_API int nq_low_bits(int n_bits, int h_bits, int compensate);
+
+/* Size of one packed row / of a whole packed tensor in bytes (host, pure).  -1 on bad arguments. */
+NQ_API int64_t nq_packed_row_bytes(int64_t cols, int bits);
+NQ_API int64_t nq_packed_bytes(int64_t rows, int64_t cols, int bits);
+
+/*
+ * Decomposition -- Eq. 5, Eq. 6, Algorithm 1 step 2, Eq. 10 and the compensation subsection.
+ * Per element: w_high = clip(round(w_int / 2^l)) to INTh, where the rounding is DOWN (the
+ * RightShift of Eq. 6) where mask == 0 and UP where mask != 0 (an exact multiple of 2^l is left
+ * alone); w_low = w_int - w_high * 2^l, clipped to l bits when compensate == 0.
+ *   w_int (device)  int8 [rows, cols], row pitch ld_w elements (>= cols)
+ *   mask  (device)  uint8 [rows, cols], same pitch: the given adaptive-rounding decision
+ *   packed_high, packed_low (device, out)  sliced tensors of h_bits and nq_low_bits() bits
+ * Fast path when w_int, mask are 16-byte aligned and ld_w is a multiple of 16; otherwise a slower
+ * byte-wise path is taken (same results).
+ */
+NQ_API int nq_decompose(const int8_t *w_int, const uint8_t *mask, int64_t rows, int64_t cols, int64_t ld_w,
+                 int n_bits, int h_bits, int compensate,
+                 void *packed_high, void *packed_low, void *stream);
+
+/*
+ * Recomposition / page-in -- Eq. 5 read as the upgrade of "Nesting Mechanism of Decomposed
+ * Weights": w_int = clip_INTn(w_high * 2^l + w_low), a shift and an ADD of the sign-extended low
+ * field.  Output int8 [rows, cols] with row pitch ld_out elements (device, out).
+ */
+NQ_API int nq_recompose(const void *packed_high, const void *packed_low, int64_t rows, int64_t cols,
+                 int n_bits, int h_bits, int compensate,
+                 int8_t *w_int_out, int64_t ld_out, void *stream);
+
+/*
+ * Drop-low / page-out -- the downgrade of the same subsection.  The full-bit resident state is
+ * {w_int, packed_low}; this derives packed_high = (w_int - w_low) / 2^l from it (no mask needed),
+ * after which the caller may free w_int and packed_low.
+ */
+NQ_API int nq_drop_low(const int8_t *w_int, int64_t ld_w, const void *packed_low, int64_t rows, int64_t cols,
+                int n_bits, int h_bits, int compensate,
+                void *packed_high_out, void *stream);
+
+/* Test aids: a sliced tensor of `bits`-bit fields <-> sign-extended int8 values. */
+NQ_API int nq_unpack(const void *packed, int bits, int64_t rows, int64_t cols,
+              int8_t *out, int64_t ld_out, void *stream);
+NQ_API int nq_pack(const int8_t *values, int64_t ld, int bits, int64_t rows, int64_t cols,
+            void *packed_out, void *stream);
+
+/*
+ * Whole-model page-in / page-out in ONE launch.  A model is a list of tensors; the caller builds
+ * the list once with nq_batch_plan and then switches the model with a single call.
+ *   descs (host)   count entries
+ *   table (device) at least nq_batch_table_bytes(count) bytes, 16-byte aligned; filled by
+ *                  nq_batch_plan with a copy queued on `stream`
+ *   total_units    work-item count nq_batch_plan reports; pass it back to the batched calls
+ * Every tensor of a batch shares (n_bits, h_bits, compensate).  w_int must be 16-byte aligned with
+ * ld a multiple of 16 for every tensor of a batch (NQ_ERR_ALIGNMENT otherwise).
+ */
+typedef struct {
+    int64_t rows, cols, ld;   /* ld: row pitch of w_int in elements */
+    void *packed_high;        /* (device) */
+    void *packed_low;         /* (device) */
+    int8_t *w_int;            /* (device) */
+} nq_tensor_desc;
+
+NQ_API int64_t nq_batch_table_bytes(int count);
+NQ_API int nq_batch_plan(const nq_tensor_desc *descs, int count, void *table, int64_t table_bytes,
+                  int64_t *total_units_out, void *stream);
+NQ_API int nq_recompose_batched(const void *table, int count, int64_t total_units,
+                         int n_bits, int h_bits, int compensate, void *stream);
+NQ_API int nq_drop_low_batched(const void *table, int count, int64_t total_units,
+                        int n_bits, int h_bits, int compensate, void *stream);
+
+/*
+ * Full-bit GEMM -- the integer layer on the recomposed weights with the dequantisation of Eq. 2:
+ *   acc[m, j] = sum_k X[m, k] * W[j, k]                       (int32, exact)
+ *   Y[m, j]   = fl(float(acc[m, j]) * fl(act_scale * w_scale[j]))  (+ bias[j], one more rounding)
+ *   X (device) int8 [M, K] pitch ldx;  W (device) int8 [N, K] pitch ldw;  both 16-byte aligned with
+ *   pitches that are multiples of 16.  w_scale (device) fp32 [N]; bias (device) fp32 [N] or NULL.
+ *   acc_out (device, out) int32 [M, N] pitch ld_acc, or NULL.  Y (device, out) [M, N] pitch ldy of
+ *   y_dtype, or NULL.  At least one of acc_out, Y must be given.  Y and acc_out 16-byte aligned,
+ *   pitches multiples of 4 elements.  K < 2^17 so that the int32 accumulator cannot overflow.
+ */
+NQ_API int nq_gemm_full(const int8_t *X, int64_t ldx, const int8_t *W, int64_t ldw,
+                 const float *w_scale, float act_scale, const float *bias,
+                 int64_t M, int64_t N, int64_t K,
+                 int32_t *acc_out, int64_t ld_acc, void *Y, int64_t ldy, int y_dtype, void *stream);
+
+/*
+ * Part-bit GEMM -- the same layer on w_high alone, unpacked from the sliced tensor inside the
+ * kernel, with the inflated scale of Eq. 9:
+ *   acc[m, j] = sum_k X[m, k] * w_high[j, k];   Y = fl(float(acc) * fl(fl(act_scale*w_scale[j]) * 2^l))
+ *   packed_high (device) sliced [N, K] tensor of h_bits fields, h_bits in [2, 7] here.
+ */
+NQ_API int nq_gemm_part(const int8_t *X, int64_t ldx, const void *packed_high, int n_bits, int h_bits,
+                 const float *w_scale, float act_scale, const float *bias,
+                 int64_t M, int64_t N, int64_t K,
+                 int32_t *acc_out, int64_t ld_acc, void *Y, int64_t ldy, int y_dtype, void *stream);
+
+/*
+ * Implicit-GEMM convolution on the nested weights, zero padding (the zero-point is 0):
+ *   acc[b, p, q, co] = sum_{r, s, ci} x[b, p*stride - pad + r, q*stride - pad + s, ci] * w[co, r, s, ci]
+ *   Y = dequantisation as in nq_gemm_full (part_bit == 0) or nq_gemm_part (part_bit != 0).
+ *   X (device) int8, NHWC [B, H, W, Cin] when x_nchw == 0, NCHW [B, Cin, H, W] when x_nchw != 0 (then
+ *     a transposing pre-pass writes an NHWC copy into the workspace).
+ *   Wt (device) weights as a [Cout, K] matrix with K = R*S*Cin in (r, s, ci) order (OHWI):
+ *     int8 with row pitch ldw (a multiple of 16, >= K) when part_bit == 0, the sliced h_bits tensor
+ *     of that matrix when part_bit != 0 (ldw ignored).
+ *   acc_out / Y: NHWC, i.e. the [M = B*Ho*Wo, N = Cout] matrix, dense.
+ *   workspace (device): nq_conv_workspace_bytes(desc) bytes, 1024-byte aligned.
+ */
+typedef struct {
+    int32_t B, Cin, H, W, Cout, R, S, stride, pad;
+    int32_t x_nchw;
+} nq_conv_desc;
+
+NQ_API int64_t nq_conv_workspace_bytes(const nq_conv_desc *desc);
+NQ_API int nq_conv_implicit_gemm(const int8_t *X, const void *Wt, int64_t ldw, int part_bit, int n_bits, int h_bits,
+                          const nq_conv_desc *desc, const float *w_scale, float act_scale,
+                          const float *bias, int32_t *acc_out, void *Y, int y_dtype,
+                          void *workspace, int64_t workspace_bytes, void *stream);
+
+/*
+ * Every on-device wait in the GEMM / convolution kernels is bounded.  If one expires the kernel
+ * records it and returns instead of hanging.  This call synchronises `stream`, reads and clears
+ * the record of the current device: returns NQ_OK, NQ_ERR_TIMEOUT (with *where_out = an internal
+ * code of the wait that gave up) or NQ_ERR_CUDA.
+ */
+NQ_API int nq_device_status(void *stream, int *where_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NQ_H_ */

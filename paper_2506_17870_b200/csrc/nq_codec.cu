@@ -1,0 +1,482 @@
+// Bandwidth-bound codec kernels: decomposition, recomposition (page-in), drop-low (page-out) and
+// the plain pack / unpack test aids, all on the sliced sub-byte layout described in nq.h.
+//
+// Work unit: 32 consecutive elements of one row = eight 32-bit words of int8 on the unpacked side
+// and, per slice of width s, s words on the packed side.  One thread owns one unit at a time and
+// keeps it in registers as eight "top-aligned" words T[q]: byte lane i of T[q] holds the k-bit
+// field of element 4q+i in its TOP k bits.  In that form every slice is a fixed bit range of every
+// byte, so moving between T and the slices is a mask, a shift and an OR per word -- four elements
+// per instruction -- and the nesting arithmetic (Eq. 5, 6, 10) is done on four bytes at a time.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "../../include/nq.h"
+#include "nq_internal.cuh"
+
+namespace {
+
+constexpr uint32_t H4 = 0x80808080u;
+constexpr uint32_t L7 = 0x7f7f7f7fu;
+
+__device__ __forceinline__ uint32_t rep8(uint32_t b) { return (b & 0xffu) * 0x01010101u; }
+
+// per-byte wrapping add / subtract, unsigned saturating subtract
+__device__ __forceinline__ uint32_t add4(uint32_t a, uint32_t b) {
+    return ((a & L7) + (b & L7)) ^ ((a ^ b) & H4);
+}
+__device__ __forceinline__ uint32_t sub4(uint32_t a, uint32_t b) {
+    return ((a | H4) - (b & L7)) ^ ((a ^ ~b) & H4);
+}
+__device__ __forceinline__ uint32_t subsat_u4(uint32_t a, uint32_t b) {
+    uint32_t d = sub4(a, b);
+    uint32_t borrow = ((~a & b) | (~(a ^ b) & d)) & H4;   // borrow out of each byte
+    uint32_t kill = (borrow >> 7) * 0xffu;
+    return d & ~kill;
+}
+// 1 in every byte that is non-zero
+__device__ __forceinline__ uint32_t nonzero4(uint32_t x) {
+    return ((((x & L7) + L7) | x) & H4) >> 7;
+}
+
+// ---------------------------------------------------------------------------------------------
+// packed side: one unit <-> eight top-aligned words
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void load_unit_top(const uint8_t* __restrict__ group, int unit, int bits,
+                                              uint32_t (&T)[8]) {
+    if (bits == 8) {
+        const uint4* p = reinterpret_cast<const uint4*>(group + unit * 32);
+        uint4 a = __ldg(p), b = __ldg(p + 1);
+        T[0] = a.x; T[1] = a.y; T[2] = a.z; T[3] = a.w; T[4] = b.x; T[5] = b.y; T[6] = b.z; T[7] = b.w;
+        return;
+    }
+#pragma unroll
+    for (int q = 0; q < 8; ++q) T[q] = 0;
+    int off = 0, used = 0;
+    if (bits & 4) {
+        uint4 w = __ldg(reinterpret_cast<const uint4*>(group + unit * 16));
+        T[0] = w.x & 0xf0f0f0f0u; T[1] = (w.x << 4) & 0xf0f0f0f0u;
+        T[2] = w.y & 0xf0f0f0f0u; T[3] = (w.y << 4) & 0xf0f0f0f0u;
+        T[4] = w.z & 0xf0f0f0f0u; T[5] = (w.z << 4) & 0xf0f0f0f0u;
+        T[6] = w.w & 0xf0f0f0f0u; T[7] = (w.w << 4) & 0xf0f0f0f0u;
+        off = 64; used = 4;
+    }
+    if (bits & 2) {
+        uint2 w = __ldg(reinterpret_cast<const uint2*>(group + off + unit * 8));
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            uint32_t word = (q < 4) ? w.x : w.y;
+            T[q] |= ((word << (2 * (q & 3))) & 0xc0c0c0c0u) >> used;
+        }
+        off += 32; used += 2;
+    }
+    if (bits & 1) {
+        uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(group + off + unit * 4));
+#pragma unroll
+        for (int q = 0; q < 8; ++q) T[q] |= ((w << q) & H4) >> used;
+    }
+}
+
+__device__ __forceinline__ void store_unit_top(uint8_t* __restrict__ group, int unit, int bits,
+                                               const uint32_t (&T)[8]) {
+    if (bits == 8) {
+        uint4* p = reinterpret_cast<uint4*>(group + unit * 32);
+        p[0] = make_uint4(T[0], T[1], T[2], T[3]);
+        p[1] = make_uint4(T[4], T[5], T[6], T[7]);
+        return;
+    }
+    int off = 0, used = 0;
+    if (bits & 4) {
+        uint4 w;
+        w.x = (T[0] & 0xf0f0f0f0u) | ((T[1] >> 4) & 0x0f0f0f0fu);
+        w.y = (T[2] & 0xf0f0f0f0u) | ((T[3] >> 4) & 0x0f0f0f0fu);
+        w.z = (T[4] & 0xf0f0f0f0u) | ((T[5] >> 4) & 0x0f0f0f0fu);
+        w.w = (T[6] & 0xf0f0f0f0u) | ((T[7] >> 4) & 0x0f0f0f0fu);
+        *reinterpret_cast<uint4*>(group + unit * 16) = w;
+        off = 64; used = 4;
+    }
+    if (bits & 2) {
+        uint2 w = make_uint2(0u, 0u);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            uint32_t piece = ((T[q] << used) & 0xc0c0c0c0u) >> (2 * (q & 3));
+            if (q < 4) w.x |= piece; else w.y |= piece;
+        }
+        *reinterpret_cast<uint2*>(group + off + unit * 8) = w;
+        off += 32; used += 2;
+    }
+    if (bits & 1) {
+        uint32_t w = 0;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) w |= ((T[q] << used) & H4) >> q;
+        *reinterpret_cast<uint32_t*>(group + off + unit * 4) = w;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// unpacked side: 32 int8 of one row <-> eight words, with a byte-wise path for ragged / unaligned rows
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void load_unit_i8(const int8_t* __restrict__ row, int64_t c0, int64_t cols,
+                                             bool vec_ok, uint32_t (&V)[8]) {
+    if (vec_ok && c0 + 32 <= cols) {
+        const uint4* p = reinterpret_cast<const uint4*>(row + c0);
+        uint4 a = __ldg(p), b = __ldg(p + 1);
+        V[0] = a.x; V[1] = a.y; V[2] = a.z; V[3] = a.w; V[4] = b.x; V[5] = b.y; V[6] = b.z; V[7] = b.w;
+    } else {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            uint32_t w = 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                int64_t c = c0 + q * 4 + i;
+                uint32_t b = (c < cols) ? (uint32_t)(uint8_t)row[c] : 0u;
+                w |= b << (8 * i);
+            }
+            V[q] = w;
+        }
+    }
+}
+
+__device__ __forceinline__ void store_unit_i8(int8_t* __restrict__ row, int64_t c0, int64_t cols,
+                                              bool vec_ok, const uint32_t (&V)[8]) {
+    if (vec_ok && c0 + 32 <= cols) {
+        uint4* p = reinterpret_cast<uint4*>(row + c0);
+        p[0] = make_uint4(V[0], V[1], V[2], V[3]);
+        p[1] = make_uint4(V[4], V[5], V[6], V[7]);
+    } else {
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                int64_t c = c0 + q * 4 + i;
+                if (c < cols) row[c] = (int8_t)((V[q] >> (8 * i)) & 0xffu);
+            }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// the nesting arithmetic on four bytes at a time.  "Biased" means value + 2^(n-1), an unsigned
+// n-bit number; in that domain w_high + 2^(h-1) is simply the top h bits.
+// ---------------------------------------------------------------------------------------------
+struct Nest {
+    int n, h, l, lb, comp;
+    uint32_t bias, mask_n, mask_h, mask_l, mask_lb, bit_l;
+    __device__ Nest(int n_, int h_, int comp_) : n(n_), h(h_), l(n_ - h_), lb(n_ - h_ + (comp_ ? 1 : 0)), comp(comp_) {
+        bias = rep8(1u << (n - 1));
+        mask_n = rep8((1u << n) - 1u);
+        mask_h = rep8((1u << h) - 1u);
+        mask_l = rep8((1u << l) - 1u);
+        mask_lb = rep8((1u << lb) - 1u);
+        bit_l = rep8(1u << l);
+    }
+};
+
+// Eq. 6 with the mask-given rounding, then Eq. 10 / compensation.  V, M: int8 weights and mask bytes.
+__device__ __forceinline__ void decompose_word(const Nest& N, uint32_t V, uint32_t M, uint32_t& Thi, uint32_t& Tlo) {
+    uint32_t wu = (V ^ N.bias) & N.mask_n;                 // w + 2^(n-1)
+    uint32_t down = (wu >> N.l) & N.mask_h;                // floor(w / 2^l) + 2^(h-1)
+    uint32_t rem = wu & N.mask_l;
+    uint32_t up = nonzero4(rem) & nonzero4(M);             // round up only off a multiple of 2^l
+    uint32_t whb = down + up;                              // <= 2^h per byte: no carry between bytes
+    whb -= (whb >> N.h) & 0x01010101u;                     // clip to 2^h - 1 (max_high, biased)
+    Thi = ((whb ^ rep8(1u << (N.h - 1))) & N.mask_h) << (8 - N.h);
+    // w_low = w - w_high * 2^l; modulo 2^(l+1) that is the low l bits of w plus one borrow bit
+    uint32_t lo = (wu ^ (whb << N.l)) & rep8((2u << N.l) - 1u);
+    if (!N.comp) {
+        // clip to [-2^(l-1), 2^(l-1) - 1]: in the domain lo + 2^l that is [2^(l-1), 3*2^(l-1) - 1]
+        uint32_t lob = lo ^ N.bit_l;
+        uint32_t half = 1u << (N.l - 1);
+        lob = __vminu4(__vmaxu4(lob, rep8(half)), rep8(3u * half - 1u));
+        lo = lob & N.mask_l;
+    }
+    Tlo = lo << (8 - N.lb);
+}
+
+// Eq. 5: shift, add the signed low field, clip to INTn.  Returns int8 bytes.
+__device__ __forceinline__ uint32_t recompose_word(const Nest& N, uint32_t Thi, uint32_t Tlo) {
+    uint32_t x = ((Thi >> (8 - N.n)) & N.mask_n) ^ N.bias;     // (w_high + 2^(h-1)) << l
+    uint32_t lo = (Tlo >> (8 - N.lb)) & N.mask_lb;
+    uint32_t a, s;
+    if (N.comp) {          // l+1-bit field: low l bits drop in, the sign bit subtracts 2^l
+        a = x | (lo & N.mask_l);
+        s = lo & N.bit_l;
+    } else {               // l-bit field: lo + 2^(l-1) drops in, then 2^(l-1) comes off
+        uint32_t half = rep8(1u << (N.l - 1));
+        a = x | (lo ^ half);
+        s = half;
+    }
+    uint32_t wu = subsat_u4(a, s);                              // the only clip that can bind is the lower one
+    return sub4(wu, N.bias);
+}
+
+// (w_int - w_low) / 2^l as an h-bit field
+__device__ __forceinline__ uint32_t drop_low_word(const Nest& N, uint32_t V, uint32_t Tlo) {
+    uint32_t lo = (Tlo >> (8 - N.lb)) & N.mask_lb;
+    uint32_t m = rep8(1u << (N.lb - 1));
+    uint32_t lo_signed = sub4(lo ^ m, m);
+    uint32_t d = sub4(V, lo_signed);
+    return ((d >> N.l) & N.mask_h) << (8 - N.h);
+}
+
+__device__ __forceinline__ uint32_t values_to_top(uint32_t V, int bits) {
+    return (V << (8 - bits)) & rep8(0xffu << (8 - bits));
+}
+__device__ __forceinline__ uint32_t top_to_values(uint32_t T, int bits) {
+    if (bits == 8) return T;
+    uint32_t x = (T >> (8 - bits)) & rep8((1u << bits) - 1u);
+    uint32_t m = rep8(1u << (bits - 1));
+    return sub4(x ^ m, m);
+}
+
+// ---------------------------------------------------------------------------------------------
+// kernels.  A tensor is rows * groups_per_row * 4 units; the grid strides over units.
+// ---------------------------------------------------------------------------------------------
+struct TensorView {
+    int64_t rows, cols, ld;
+    uint8_t* hi;
+    uint8_t* lo;
+    int8_t* w;
+    const uint8_t* mask;
+};
+
+enum Op { OP_DECOMPOSE = 0, OP_RECOMPOSE = 1, OP_DROP_LOW = 2, OP_UNPACK = 3, OP_PACK = 4 };
+
+template <int OP>
+__device__ __forceinline__ void do_unit(const TensorView& t, int64_t unit_index, const Nest& N, int bits) {
+    const int64_t units_per_row = ((t.cols + 127) / 128) * 4;
+    const int64_t row = unit_index / units_per_row;
+    const int64_t ur = unit_index - row * units_per_row;
+    const int64_t group = ur >> 2;
+    const int unit = (int)(ur & 3);
+    const int64_t c0 = ur * 32;
+    const bool vec_ok = ((t.ld & 15) == 0) && ((reinterpret_cast<uintptr_t>(t.w) & 15) == 0) &&
+                        (OP != OP_DECOMPOSE || (reinterpret_cast<uintptr_t>(t.mask) & 15) == 0);
+    int8_t* wrow = t.w + row * t.ld;
+    uint32_t A[8], Bv[8];
+    if (OP == OP_DECOMPOSE) {
+        uint8_t* ghi = t.hi + (row * (units_per_row >> 2) + group) * 16 * N.h;
+        uint8_t* glo = t.lo + (row * (units_per_row >> 2) + group) * 16 * N.lb;
+        load_unit_i8(wrow, c0, t.cols, vec_ok, A);
+        load_unit_i8(reinterpret_cast<const int8_t*>(t.mask) + row * t.ld, c0, t.cols, vec_ok, Bv);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) decompose_word(N, A[q], Bv[q], A[q], Bv[q]);
+        store_unit_top(ghi, unit, N.h, A);
+        store_unit_top(glo, unit, N.lb, Bv);
+    } else if (OP == OP_RECOMPOSE) {
+        const uint8_t* ghi = t.hi + (row * (units_per_row >> 2) + group) * 16 * N.h;
+        const uint8_t* glo = t.lo + (row * (units_per_row >> 2) + group) * 16 * N.lb;
+        load_unit_top(ghi, unit, N.h, A);
+        load_unit_top(glo, unit, N.lb, Bv);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) A[q] = recompose_word(N, A[q], Bv[q]);
+        store_unit_i8(wrow, c0, t.cols, vec_ok, A);
+    } else if (OP == OP_DROP_LOW) {
+        uint8_t* ghi = t.hi + (row * (units_per_row >> 2) + group) * 16 * N.h;
+        const uint8_t* glo = t.lo + (row * (units_per_row >> 2) + group) * 16 * N.lb;
+        load_unit_i8(wrow, c0, t.cols, vec_ok, A);
+        load_unit_top(glo, unit, N.lb, Bv);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) A[q] = drop_low_word(N, A[q], Bv[q]);
+        store_unit_top(ghi, unit, N.h, A);
+    } else if (OP == OP_UNPACK) {
+        const uint8_t* g = t.hi + (row * (units_per_row >> 2) + group) * 16 * bits;
+        load_unit_top(g, unit, bits, A);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) A[q] = top_to_values(A[q], bits);
+        store_unit_i8(wrow, c0, t.cols, vec_ok, A);
+    } else {
+        uint8_t* g = t.hi + (row * (units_per_row >> 2) + group) * 16 * bits;
+        load_unit_i8(wrow, c0, t.cols, vec_ok, A);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) A[q] = values_to_top(A[q], bits);
+        store_unit_top(g, unit, bits, A);
+    }
+}
+
+template <int OP>
+__global__ void __launch_bounds__(256) codec_kernel(TensorView t, int64_t total_units, int n, int h, int comp, int bits) {
+    const Nest N(n, h, comp);
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < total_units; u += stride)
+        do_unit<OP>(t, u, N, bits);
+}
+
+// one launch over a whole model: table entries carry the running unit count
+struct BatchEntry {
+    int64_t rows, cols, ld;
+    uint8_t* hi;
+    uint8_t* lo;
+    int8_t* w;
+    int64_t first_unit;     // units of all earlier tensors
+    int64_t pad_;
+};
+static_assert(sizeof(BatchEntry) == 64, "table entry is 64 bytes");
+
+template <int OP>
+__global__ void __launch_bounds__(256) codec_batched_kernel(const BatchEntry* __restrict__ table, int count,
+                                                            int64_t total_units, int n, int h, int comp) {
+    const Nest N(n, h, comp);
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < total_units; u += stride) {
+        int lo = 0, hi = count - 1;                 // last entry whose first_unit <= u
+        while (lo < hi) {
+            int mid = (lo + hi + 1) >> 1;
+            if (__ldg(&table[mid].first_unit) <= u) lo = mid; else hi = mid - 1;
+        }
+        const BatchEntry* e = table + lo;
+        TensorView t;
+        t.rows = __ldg(&e->rows); t.cols = __ldg(&e->cols); t.ld = __ldg(&e->ld);
+        t.hi = e->hi; t.lo = e->lo; t.w = e->w; t.mask = nullptr;
+        do_unit<OP>(t, u - __ldg(&e->first_unit), N, 0);
+    }
+}
+
+inline int launch_blocks(int64_t total_units) {
+    int64_t need = (total_units + 255) / 256;
+    int64_t cap = (int64_t)nq::sm_count() * 8 * 4;
+    return (int)(need < cap ? need : cap);
+}
+
+inline bool nest_ok(int n, int h) { return n >= 2 && n <= 8 && h >= 1 && h < n; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+template <int OP>
+int run_single(TensorView t, int n, int h, int comp, int bits, void* stream) {
+    if (t.rows == 0 || t.cols == 0) return NQ_OK;
+    int64_t total = t.rows * ((t.cols + 127) / 128) * 4;
+    codec_kernel<OP><<<launch_blocks(total), 256, 0, (cudaStream_t)stream>>>(t, total, n, h, comp, bits);
+    return cudaGetLastError() == cudaSuccess ? NQ_OK : NQ_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+int nq_low_bits(int n_bits, int h_bits, int compensate) {
+    if (!nest_ok(n_bits, h_bits)) return -1;
+    return n_bits - h_bits + (compensate ? 1 : 0);
+}
+
+int64_t nq_packed_row_bytes(int64_t cols, int bits) {
+    if (cols < 0 || bits < 1 || bits > 8) return -1;
+    return ((cols + 127) / 128) * 16 * bits;
+}
+
+int64_t nq_packed_bytes(int64_t rows, int64_t cols, int bits) {
+    if (rows < 0) return -1;
+    int64_t r = nq_packed_row_bytes(cols, bits);
+    return r < 0 ? -1 : r * rows;
+}
+
+int nq_decompose(const int8_t* w_int, const uint8_t* mask, int64_t rows, int64_t cols, int64_t ld_w,
+                 int n_bits, int h_bits, int compensate, void* packed_high, void* packed_low, void* stream) {
+    if (rows < 0 || cols < 0) return NQ_ERR_INVALID_ARG;
+    if (!nest_ok(n_bits, h_bits)) return NQ_ERR_UNSUPPORTED;
+    if (rows == 0 || cols == 0) return NQ_OK;
+    if (!w_int || !mask || !packed_high || !packed_low || ld_w < cols) return NQ_ERR_INVALID_ARG;
+    if (!aligned16(packed_high) || !aligned16(packed_low)) return NQ_ERR_ALIGNMENT;
+    TensorView t{rows, cols, ld_w, (uint8_t*)packed_high, (uint8_t*)packed_low, (int8_t*)w_int, mask};
+    return run_single<OP_DECOMPOSE>(t, n_bits, h_bits, compensate ? 1 : 0, 0, stream);
+}
+
+int nq_recompose(const void* packed_high, const void* packed_low, int64_t rows, int64_t cols,
+                 int n_bits, int h_bits, int compensate, int8_t* w_int_out, int64_t ld_out, void* stream) {
+    if (rows < 0 || cols < 0) return NQ_ERR_INVALID_ARG;
+    if (!nest_ok(n_bits, h_bits)) return NQ_ERR_UNSUPPORTED;
+    if (rows == 0 || cols == 0) return NQ_OK;
+    if (!w_int_out || !packed_high || !packed_low || ld_out < cols) return NQ_ERR_INVALID_ARG;
+    if (!aligned16(packed_high) || !aligned16(packed_low)) return NQ_ERR_ALIGNMENT;
+    TensorView t{rows, cols, ld_out, (uint8_t*)packed_high, (uint8_t*)packed_low, w_int_out, nullptr};
+    return run_single<OP_RECOMPOSE>(t, n_bits, h_bits, compensate ? 1 : 0, 0, stream);
+}
+
+int nq_drop_low(const int8_t* w_int, int64_t ld_w, const void* packed_low, int64_t rows, int64_t cols,
+                int n_bits, int h_bits, int compensate, void* packed_high_out, void* stream) {
+    if (rows < 0 || cols < 0) return NQ_ERR_INVALID_ARG;
+    if (!nest_ok(n_bits, h_bits)) return NQ_ERR_UNSUPPORTED;
+    if (rows == 0 || cols == 0) return NQ_OK;
+    if (!w_int || !packed_high_out || !packed_low || ld_w < cols) return NQ_ERR_INVALID_ARG;
+    if (!aligned16(packed_high_out) || !aligned16(packed_low)) return NQ_ERR_ALIGNMENT;
+    TensorView t{rows, cols, ld_w, (uint8_t*)packed_high_out, (uint8_t*)packed_low, (int8_t*)w_int, nullptr};
+    return run_single<OP_DROP_LOW>(t, n_bits, h_bits, compensate ? 1 : 0, 0, stream);
+}
+
+int nq_unpack(const void* packed, int bits, int64_t rows, int64_t cols, int8_t* out, int64_t ld_out, void* stream) {
+    if (rows < 0 || cols < 0) return NQ_ERR_INVALID_ARG;
+    if (bits < 1 || bits > 8) return NQ_ERR_UNSUPPORTED;
+    if (rows == 0 || cols == 0) return NQ_OK;
+    if (!packed || !out || ld_out < cols) return NQ_ERR_INVALID_ARG;
+    if (!aligned16(packed)) return NQ_ERR_ALIGNMENT;
+    TensorView t{rows, cols, ld_out, (uint8_t*)packed, nullptr, out, nullptr};
+    return run_single<OP_UNPACK>(t, 8, 4, 1, bits, stream);
+}
+
+int nq_pack(const int8_t* values, int64_t ld, int bits, int64_t rows, int64_t cols, void* packed_out, void* stream) {
+    if (rows < 0 || cols < 0) return NQ_ERR_INVALID_ARG;
+    if (bits < 1 || bits > 8) return NQ_ERR_UNSUPPORTED;
+    if (rows == 0 || cols == 0) return NQ_OK;
+    if (!values || !packed_out || ld < cols) return NQ_ERR_INVALID_ARG;
+    if (!aligned16(packed_out)) return NQ_ERR_ALIGNMENT;
+    TensorView t{rows, cols, ld, (uint8_t*)packed_out, nullptr, (int8_t*)values, nullptr};
+    return run_single<OP_PACK>(t, 8, 4, 1, bits, stream);
+}
+
+int64_t nq_batch_table_bytes(int count) {
+    if (count < 0) return -1;
+    return (int64_t)(count > 0 ? count : 1) * (int64_t)sizeof(BatchEntry);
+}
+
+int nq_batch_plan(const nq_tensor_desc* descs, int count, void* table, int64_t table_bytes,
+                  int64_t* total_units_out, void* stream) {
+    if (count < 0 || (count > 0 && !descs) || !table || !total_units_out) return NQ_ERR_INVALID_ARG;
+    if (table_bytes < nq_batch_table_bytes(count)) return NQ_ERR_WORKSPACE;
+    if (!aligned16(table)) return NQ_ERR_ALIGNMENT;
+    std::vector<BatchEntry> host((size_t)count);
+    int64_t units = 0;
+    for (int i = 0; i < count; ++i) {
+        const nq_tensor_desc& d = descs[i];
+        if (d.rows < 0 || d.cols < 0 || d.ld < d.cols) return NQ_ERR_INVALID_ARG;
+        if (d.rows > 0 && d.cols > 0) {
+            if (!d.packed_high || !d.packed_low || !d.w_int) return NQ_ERR_INVALID_ARG;
+            if (!aligned16(d.packed_high) || !aligned16(d.packed_low) || !aligned16(d.w_int) || (d.ld & 15))
+                return NQ_ERR_ALIGNMENT;
+        }
+        BatchEntry& e = host[i];
+        e.rows = d.rows; e.cols = d.cols; e.ld = d.ld;
+        e.hi = (uint8_t*)d.packed_high; e.lo = (uint8_t*)d.packed_low; e.w = d.w_int;
+        e.first_unit = units; e.pad_ = 0;
+        units += d.rows * ((d.cols + 127) / 128) * 4;
+    }
+    *total_units_out = units;
+    if (count == 0) return NQ_OK;
+    // the source is pageable host memory: the runtime stages it before this call returns
+    cudaError_t err = cudaMemcpyAsync(table, host.data(), (size_t)count * sizeof(BatchEntry),
+                                      cudaMemcpyHostToDevice, (cudaStream_t)stream);
+    return err == cudaSuccess ? NQ_OK : NQ_ERR_CUDA;
+}
+
+static int run_batched(int op, const void* table, int count, int64_t units, int n, int h, int comp, void* stream) {
+    if (count < 0 || units < 0 || !table) return NQ_ERR_INVALID_ARG;
+    if (!nest_ok(n, h)) return NQ_ERR_UNSUPPORTED;
+    if (count == 0 || units == 0) return NQ_OK;
+    const BatchEntry* entries = reinterpret_cast<const BatchEntry*>(table);
+    int blocks = launch_blocks(units);
+    if (op == OP_RECOMPOSE)
+        codec_batched_kernel<OP_RECOMPOSE><<<blocks, 256, 0, (cudaStream_t)stream>>>(entries, count, units, n, h, comp);
+    else
+        codec_batched_kernel<OP_DROP_LOW><<<blocks, 256, 0, (cudaStream_t)stream>>>(entries, count, units, n, h, comp);
+    return cudaGetLastError() == cudaSuccess ? NQ_OK : NQ_ERR_CUDA;
+}
+
+int nq_recompose_batched(const void* table, int count, int64_t total_units, int n_bits, int h_bits, int compensate,
+                         void* stream) {
+    return run_batched(OP_RECOMPOSE, table, count, total_units, n_bits, h_bits, compensate ? 1 : 0, stream);
+}
+
+int nq_drop_low_batched(const void* table, int count, int64_t total_units, int n_bits, int h_bits, int compensate,
+                        void* stream) {
+    return run_batched(OP_DROP_LOW, table, count, total_units, n_bits, h_bits, compensate ? 1 : 0, stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,375 @@
+// The INT8 contraction kernel shared by the GEMM and the implicit-GEMM convolution.
+//
+//   acc[m, j] = sum_k A[m, k] * B[j, k]   (int8 x int8 -> int32 on the tcgen05 tensor cores)
+//   Y[m, j]   = float(acc) * scale[j] (+ bias[j])       fused epilogue, fp32 or bf16
+//
+// One persistent CTA per SM walks a list of 128 x BN output tiles.  Roles (warp-specialised):
+//   warp 0      TMA producer: A tile (128 rows x 128 B) and B tile (BN rows x 128 B, or the packed
+//               INTh tile in part-bit mode) into a ring of shared-memory stages
+//   warp 1      MMA issuer: one thread issues four tcgen05.mma kind::i8 (K = 32 each) per stage into
+//               a TMEM accumulator; owns the TMEM allocation
+//   warps 2-5   epilogue: tcgen05.ld the accumulator (each warp its 32-lane quarter), scale, store.
+//               Two accumulators alternate so the epilogue of tile i overlaps the MMAs of tile i+1
+//   warps 6-9   (part-bit only) unpackers: expand packed INTh fields into the swizzled int8 B tile.
+//               The field goes to the TOP h bits of the byte, i.e. the byte is w_high * 2^(8-h); the
+//               accumulator is then 2^(8-h) times too large, exactly, and the epilogue takes it out
+//               (arithmetic shift for the int32 output, an exact power-of-two factor in the scale).
+// Every mbarrier wait is bounded (see mbar_wait); when one gives up every role leaves its loop,
+// the block joins, frees its TMEM and returns, and the host can read the record.
+#pragma once
+#include <cuda_bf16.h>
+
+#include "nq_sm100.cuh"
+
+namespace nq {
+
+constexpr int kBM = 128;           // tile rows (M) = TMEM lanes
+constexpr int kBK = 128;           // K bytes per stage = one 128-byte swizzle row
+constexpr int kStagesFull = 4;
+constexpr int kStagesPart = 3;
+constexpr int kPackedStages = 2;
+constexpr int kGroupM = 16;        // tile rasterisation: 16 M-tiles share a band of N-tiles
+
+struct ContractionArgs {
+    int M, N, K;
+    int m_tiles, n_tiles, k_blocks;
+    const float* w_scale;
+    const float* bias;
+    float act_scale;
+    float pow2_l;        // 2^l in part-bit mode, 1 otherwise
+    float unshift;       // 2^-(8-h) in part-bit mode, 1 otherwise (exact)
+    int acc_shift;       // 8-h in part-bit mode, 0 otherwise
+    int h_bits;          // part-bit: width of the packed field
+    int32_t* acc_out;
+    long long ld_acc;
+    void* y;
+    long long ldy;
+    int y_is_bf16;
+    unsigned int* status;
+};
+
+__host__ __device__ constexpr int a_stage_bytes() { return kBM * kBK; }
+__host__ __device__ constexpr int b_stage_bytes(int bn) { return bn * kBK; }
+
+// dynamic shared memory: [A stages][B stages][packed stages][scale + bias per epilogue warp][barriers]
+__host__ __device__ inline int contraction_smem_bytes(int bn, bool part, int h_bits) {
+    int stages = part ? kStagesPart : kStagesFull;
+    int bytes = stages * (a_stage_bytes() + b_stage_bytes(bn));
+    if (part) bytes += kPackedStages * bn * 16 * h_bits;
+    bytes += 4 * 2 * bn * (int)sizeof(float);   // scale and bias, one private copy per epilogue warp
+    bytes += 256;                       // barriers, TMEM base, abort flag
+    return bytes + 1024;                // slack to align the base to 1024 B
+}
+
+__device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, int& mt, int& nt) {
+    const int per_group = kGroupM * n_tiles;
+    const int g = tile / per_group;
+    const int first = g * kGroupM;
+    const int gsz = min(m_tiles - first, kGroupM);
+    const int local = tile - g * per_group;
+    mt = first + local % gsz;
+    nt = local / gsz;
+}
+
+// expand one 32-element unit of h-bit fields to 32 bytes, field in the top bits of each byte
+__device__ __forceinline__ void unpack_unit_top(const uint8_t* group, int unit, int bits, uint32_t (&T)[8]) {
+#pragma unroll
+    for (int q = 0; q < 8; ++q) T[q] = 0;
+    int off = 0, used = 0;
+    if (bits & 4) {
+        uint4 w = *reinterpret_cast<const uint4*>(group + unit * 16);
+        T[0] = w.x & 0xf0f0f0f0u; T[1] = (w.x << 4) & 0xf0f0f0f0u;
+        T[2] = w.y & 0xf0f0f0f0u; T[3] = (w.y << 4) & 0xf0f0f0f0u;
+        T[4] = w.z & 0xf0f0f0f0u; T[5] = (w.z << 4) & 0xf0f0f0f0u;
+        T[6] = w.w & 0xf0f0f0f0u; T[7] = (w.w << 4) & 0xf0f0f0f0u;
+        off = 64; used = 4;
+    }
+    if (bits & 2) {
+        uint2 w = *reinterpret_cast<const uint2*>(group + off + unit * 8);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            uint32_t word = (q < 4) ? w.x : w.y;
+            T[q] |= ((word << (2 * (q & 3))) & 0xc0c0c0c0u) >> used;
+        }
+        off += 32; used += 2;
+    }
+    if (bits & 1) {
+        uint32_t w = *reinterpret_cast<const uint32_t*>(group + off + unit * 4);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) T[q] |= ((w << q) & 0x80808080u) >> used;
+    }
+}
+
+template <int BN, bool PART>
+__global__ void __launch_bounds__(PART ? 320 : 192, 1)
+contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                   const ContractionArgs p) {
+    using namespace sm100;
+    constexpr int STAGES = PART ? kStagesPart : kStagesFull;
+    constexpr int A_BYTES = a_stage_bytes();
+    constexpr int B_BYTES = b_stage_bytes(BN);
+    constexpr uint32_t TMEM_COLS = (2 * BN < 32) ? 32 : 2 * BN;       // power of two >= 32
+    constexpr uint32_t IDESC = idesc_i8(kBM, BN);
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sA = smem;
+    uint8_t* sB = sA + STAGES * A_BYTES;
+    const int packed_bytes = PART ? BN * 16 * p.h_bits : 0;
+    uint8_t* sP = sB + STAGES * B_BYTES;
+    float* sScale = reinterpret_cast<float*>(sP + (PART ? kPackedStages * packed_bytes : 0));   // [4 warps][BN]
+    float* sBias = sScale + 4 * BN;                                                             // [4 warps][BN]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sBias + 4 * BN);
+    // barrier map: full[STAGES], empty[STAGES], pfull[2], pempty[2], tfull[2], tempty[2]
+    uint64_t* full = bars;
+    uint64_t* empty = full + STAGES;
+    uint64_t* pfull = empty + STAGES;
+    uint64_t* pempty = pfull + kPackedStages;
+    uint64_t* tfull = pempty + kPackedStages;
+    uint64_t* tempty = tfull + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int num_tiles = p.m_tiles * p.n_tiles;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(smem_u32(&full[s]), PART ? 1 + 4 : 1);   // producer (+ one arrival per unpack warp)
+            mbar_init(smem_u32(&empty[s]), 1);                 // tcgen05.commit
+        }
+        for (int s = 0; s < kPackedStages; ++s) {
+            mbar_init(smem_u32(&pfull[s]), 1);
+            mbar_init(smem_u32(&pempty[s]), 4);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&tfull[b]), 1);
+            mbar_init(smem_u32(&tempty[b]), 4);                // one arrival per epilogue warp
+        }
+        *abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&tmA);
+        prefetch_tensormap(&tmB);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t it = 0, pit = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+                int mt, nt;
+                tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                    const uint32_t s = it % STAGES, use = it / STAGES;
+                    if (!(ok = mbar_wait(smem_u32(&empty[s]), (use & 1) ^ 1, abort_flag, p.status, 0x10u))) break;
+                    const uint32_t fb = smem_u32(&full[s]);
+                    if (PART) {
+                        mbar_arrive_expect_tx(fb, A_BYTES);
+                        tma_load_2d(smem_u32(sA + s * A_BYTES), &tmA, kb * kBK, mt * kBM, fb);
+                        const uint32_t ps = pit % kPackedStages, puse = pit / kPackedStages;
+                        if (!(ok = mbar_wait(smem_u32(&pempty[ps]), (puse & 1) ^ 1, abort_flag, p.status, 0x11u))) break;
+                        const uint32_t pb = smem_u32(&pfull[ps]);
+                        mbar_arrive_expect_tx(pb, packed_bytes);
+                        tma_load_2d(smem_u32(sP + ps * packed_bytes), &tmB, kb * 16 * p.h_bits, nt * BN, pb);
+                        ++pit;
+                    } else {
+                        mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
+                        tma_load_2d(smem_u32(sA + s * A_BYTES), &tmA, kb * kBK, mt * kBM, fb);
+                        tma_load_2d(smem_u32(sB + s * B_BYTES), &tmB, kb * kBK, nt * BN, fb);
+                    }
+                }
+            }
+            if (!ok) {
+                // gave up: let the copies already in flight land before the block releases its shared memory
+                const long long t0 = clock64();
+                while (clock64() - t0 < (1ll << 22)) { }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            uint32_t it = 0, tl = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tl) {
+                const uint32_t buf = tl & 1, buse = tl >> 1;
+                if (!(ok = mbar_wait(smem_u32(&tempty[buf]), (buse & 1) ^ 1, abort_flag, p.status, 0x20u))) break;
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + buf * BN;
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                    const uint32_t s = it % STAGES, use = it / STAGES;
+                    if (!(ok = mbar_wait(smem_u32(&full[s]), use & 1, abort_flag, p.status, 0x21u))) break;
+                    tc_fence_after_sync();
+                    const uint64_t da = smem_desc_sw128(smem_u32(sA + s * A_BYTES));
+                    const uint64_t db = smem_desc_sw128(smem_u32(sB + s * B_BYTES));
+#pragma unroll
+                    for (int k = 0; k < kBK / 32; ++k)   // 32 bytes of K per instruction: +2 in the address field
+                        mma_i8(d_tmem, da + 2 * k, db + 2 * k, IDESC, (kb | k) != 0);
+                    mma_commit(smem_u32(&empty[s]));       // stage reusable once these MMAs have read it
+                }
+                if (ok) mma_commit(smem_u32(&tfull[buf]));   // accumulator complete
+            }
+        }
+    } else if (warp < 6) {
+        // ------------------------------------------------------------------ epilogue
+        const int quarter = warp & 3;                  // TMEM lanes this warp may read
+        uint32_t tl = 0;
+        bool ok = true;
+        const bool vec_f32 = (p.y != nullptr) && !p.y_is_bf16 && ((p.ldy & 3) == 0) &&
+                             ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
+        const bool vec_bf16 = (p.y != nullptr) && p.y_is_bf16 && ((p.ldy & 7) == 0) &&
+                              ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
+        const bool vec_acc = (p.acc_out != nullptr) && ((p.ld_acc & 3) == 0) &&
+                             ((reinterpret_cast<uintptr_t>(p.acc_out) & 15) == 0);
+        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tl) {
+            int mt, nt;
+            tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
+            const uint32_t buf = tl & 1, buse = tl >> 1;
+            const int n0 = nt * BN;
+            // per-channel factor: fl(fl(act * w_scale) * 2^l), then the exact 2^-(8-h) of the unpack.
+            // Each warp keeps a private copy, so the epilogue warps never wait on one another.
+            float* sc_w = sScale + (warp - 2) * BN;
+            float* bs_w = sBias + (warp - 2) * BN;
+            __syncwarp();
+            for (int j = lane; j < BN; j += 32) {
+                const int col = n0 + j;
+                float sc = 0.f, bs = 0.f;
+                if (col < p.N) {
+                    sc = __fmul_rn(__fmul_rn(__fmul_rn(p.act_scale, p.w_scale[col]), p.pow2_l), p.unshift);
+                    if (p.bias) bs = p.bias[col];
+                }
+                sc_w[j] = sc;
+                bs_w[j] = bs;
+            }
+            __syncwarp();
+            ok = mbar_wait(smem_u32(&tfull[buf]), buse & 1, abort_flag, p.status, 0x30u);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const long long row = (long long)mt * kBM + quarter * 32 + lane;
+            const bool row_ok = row < p.M;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld_32x32(tmem_base + buf * BN + c * 32 + ((uint32_t)(quarter * 32) << 16), r);
+                tmem_ld_wait();
+                const int col0 = n0 + c * 32;
+                if (!row_ok || col0 >= p.N) continue;
+                const float* sc = sc_w + c * 32;
+                const float* bs = bs_w + c * 32;
+                const bool full_chunk = col0 + 32 <= p.N;
+                if (p.acc_out) {
+                    int32_t* dst = p.acc_out + row * p.ld_acc + col0;
+                    if (full_chunk && vec_acc) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            *reinterpret_cast<int4*>(dst + j) =
+                                make_int4((int)r[j] >> p.acc_shift, (int)r[j + 1] >> p.acc_shift,
+                                          (int)r[j + 2] >> p.acc_shift, (int)r[j + 3] >> p.acc_shift);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (col0 + j < p.N) dst[j] = (int)r[j] >> p.acc_shift;
+                    }
+                }
+                if (p.y) {
+                    float v[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        float t = __fmul_rn(__int2float_rn((int)r[j]), sc[j]);
+                        v[j] = p.bias ? __fadd_rn(t, bs[j]) : t;
+                    }
+                    if (!p.y_is_bf16) {
+                        float* dst = reinterpret_cast<float*>(p.y) + row * p.ldy + col0;
+                        if (full_chunk && vec_f32) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4)
+                                *reinterpret_cast<float4*>(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (col0 + j < p.N) dst[j] = v[j];
+                        }
+                    } else {
+                        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.y) + row * p.ldy + col0;
+                        if (full_chunk && vec_bf16) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 8) {
+                                __nv_bfloat162 a = __floats2bfloat162_rn(v[j], v[j + 1]);
+                                __nv_bfloat162 b = __floats2bfloat162_rn(v[j + 2], v[j + 3]);
+                                __nv_bfloat162 c2 = __floats2bfloat162_rn(v[j + 4], v[j + 5]);
+                                __nv_bfloat162 d = __floats2bfloat162_rn(v[j + 6], v[j + 7]);
+                                uint4 o;
+                                o.x = *reinterpret_cast<uint32_t*>(&a);
+                                o.y = *reinterpret_cast<uint32_t*>(&b);
+                                o.z = *reinterpret_cast<uint32_t*>(&c2);
+                                o.w = *reinterpret_cast<uint32_t*>(&d);
+                                *reinterpret_cast<uint4*>(dst + j) = o;
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (col0 + j < p.N) dst[j] = __float2bfloat16_rn(v[j]);
+                        }
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tempty[buf]));
+        }
+    } else if (PART) {
+        // ------------------------------------------------------------------ unpackers (warps 6-9)
+        const int utid = threadIdx.x - 192;            // 0..127
+        uint32_t it = 0;
+        bool ok = true;
+        const int h = p.h_bits;
+        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+            for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                const uint32_t s = it % STAGES, use = it / STAGES;
+                const uint32_t ps = it % kPackedStages, puse = it / kPackedStages;
+                ok = mbar_wait(smem_u32(&pfull[ps]), puse & 1, abort_flag, p.status, 0x40u) &&
+                     mbar_wait(smem_u32(&empty[s]), (use & 1) ^ 1, abort_flag, p.status, 0x41u);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const uint8_t* src = sP + ps * packed_bytes;
+                uint8_t* dst = sB + s * B_BYTES;
+#pragma unroll 2
+                for (int task = utid; task < BN * 4; task += 128) {
+                    const int row = task >> 2, unit = task & 3;
+                    uint32_t T[8];
+                    unpack_unit_top(src + row * 16 * h, unit, h, T);
+                    uint8_t* drow = dst + row * 128;
+                    const int sw = row & 7;
+                    *reinterpret_cast<uint4*>(drow + (((2 * unit) ^ sw) << 4)) = make_uint4(T[0], T[1], T[2], T[3]);
+                    *reinterpret_cast<uint4*>(drow + (((2 * unit + 1) ^ sw) << 4)) = make_uint4(T[4], T[5], T[6], T[7]);
+                }
+                fence_proxy_async_smem();              // these writes feed tcgen05.mma (async proxy)
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(smem_u32(&full[s]));
+                    mbar_arrive(smem_u32(&pempty[ps]));
+                }
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+}  // namespace nq

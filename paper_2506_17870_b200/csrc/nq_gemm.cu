@@ -1,0 +1,143 @@
+// Host side of the nested GEMM entry points: argument checks, TMA descriptors, launch.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/nq.h"
+#include "nq_contraction.cuh"
+#include "nq_internal.cuh"
+
+namespace nq {
+
+int encode_tensor_map_2d(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t pitch_bytes,
+                         uint32_t box_inner, uint32_t box_outer, bool swizzle128) {
+    typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                 const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static EncodeFn fn = nullptr;
+    if (!fn) {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess || !sym ||
+            q != cudaDriverEntryPointSuccess)
+            return NQ_ERR_CUDA;
+        fn = reinterpret_cast<EncodeFn>(sym);
+    }
+    cuuint64_t dims[2] = {inner, outer};
+    cuuint64_t strides[1] = {pitch_bytes};
+    cuuint32_t box[2] = {box_inner, box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? NQ_OK : NQ_ERR_CUDA;
+}
+
+namespace {
+
+template <int BN, bool PART>
+int launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const ContractionArgs& a, cudaStream_t stream) {
+    const int smem = contraction_smem_bytes(BN, PART, a.h_bits);
+    static int configured[64] = {0};       // largest opt-in done so far, per device, for this instantiation
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return NQ_ERR_CUDA;
+    if (smem > configured[dev]) {
+        if (cudaFuncSetAttribute(contraction_kernel<BN, PART>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
+            cudaSuccess)
+            return NQ_ERR_CUDA;
+        configured[dev] = smem;
+    }
+    const int tiles = a.m_tiles * a.n_tiles;
+    const int grid = tiles < sm_count() ? tiles : sm_count();
+    contraction_kernel<BN, PART><<<grid, PART ? 320 : 192, smem, stream>>>(tmA, tmB, a);
+    return cudaGetLastError() == cudaSuccess ? NQ_OK : NQ_ERR_CUDA;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+}  // namespace
+
+// A is an int8 [M, K] matrix reached through tmA (built by the caller: plain 2-D for the GEMM).
+int run_contraction(const CUtensorMap& tmA, const void* Bmat, int64_t ldb, bool part, int n_bits, int h_bits,
+                    const float* w_scale, float act_scale, const float* bias, int64_t M, int64_t N, int64_t K,
+                    int32_t* acc_out, int64_t ld_acc, void* Y, int64_t ldy, int y_dtype, cudaStream_t stream) {
+    const int bn = N > 128 ? 256 : (N > 64 ? 128 : 64);
+    ContractionArgs a{};
+    a.M = (int)M; a.N = (int)N; a.K = (int)K;
+    a.m_tiles = (int)((M + kBM - 1) / kBM);
+    a.n_tiles = (int)((N + bn - 1) / bn);
+    a.k_blocks = (int)((K + kBK - 1) / kBK);
+    a.w_scale = w_scale; a.bias = bias; a.act_scale = act_scale;
+    a.acc_out = acc_out; a.ld_acc = ld_acc; a.y = Y; a.ldy = ldy; a.y_is_bf16 = (y_dtype == NQ_BF16);
+    a.status = status_word();
+    if (!a.status) return NQ_ERR_CUDA;
+    CUtensorMap tmB;
+    if (part) {
+        const int l = n_bits - h_bits;
+        a.pow2_l = (float)(1 << l);
+        a.acc_shift = 8 - h_bits;
+        a.unshift = 1.0f / (float)(1 << a.acc_shift);
+        a.h_bits = h_bits;
+        const uint64_t row_bytes = (uint64_t)a.k_blocks * 16 * h_bits;
+        int st = encode_tensor_map_2d(&tmB, Bmat, row_bytes, (uint64_t)N, row_bytes, 16 * h_bits, bn, false);
+        if (st != NQ_OK) return st;
+    } else {
+        a.pow2_l = 1.0f; a.unshift = 1.0f; a.acc_shift = 0; a.h_bits = 0;
+        int st = encode_tensor_map_2d(&tmB, Bmat, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, kBK, bn, true);
+        if (st != NQ_OK) return st;
+    }
+    if (part) {
+        if (bn == 256) return launch<256, true>(tmA, tmB, a, stream);
+        if (bn == 128) return launch<128, true>(tmA, tmB, a, stream);
+        return launch<64, true>(tmA, tmB, a, stream);
+    }
+    if (bn == 256) return launch<256, false>(tmA, tmB, a, stream);
+    if (bn == 128) return launch<128, false>(tmA, tmB, a, stream);
+    return launch<64, false>(tmA, tmB, a, stream);
+}
+
+namespace {
+
+int gemm_common(const int8_t* X, int64_t ldx, const void* Bmat, int64_t ldb, bool part, int n_bits, int h_bits,
+                const float* w_scale, float act_scale, const float* bias, int64_t M, int64_t N, int64_t K,
+                int32_t* acc_out, int64_t ld_acc, void* Y, int64_t ldy, int y_dtype, void* stream) {
+    if (M < 0 || N < 0 || K < 0) return NQ_ERR_INVALID_ARG;
+    if (y_dtype != NQ_F32 && y_dtype != NQ_BF16) return NQ_ERR_INVALID_ARG;
+    if (part && (n_bits < 2 || n_bits > 8 || h_bits < 1 || h_bits >= n_bits)) return NQ_ERR_UNSUPPORTED;
+    if (K >= (1 << 17) || M > (1ll << 30) || N > (1ll << 30)) return NQ_ERR_UNSUPPORTED;
+    if (M == 0 || N == 0) return NQ_OK;
+    if (!acc_out && !Y) return NQ_ERR_INVALID_ARG;
+    if (!w_scale && Y) return NQ_ERR_INVALID_ARG;
+    if ((acc_out && ld_acc < N) || (Y && ldy < N)) return NQ_ERR_INVALID_ARG;
+    if (K == 0) return NQ_ERR_UNSUPPORTED;
+    if (!X || !Bmat || ldx < K || (!part && ldb < K)) return NQ_ERR_INVALID_ARG;
+    if (!aligned16(X) || (ldx & 15) || !aligned16(Bmat) || (!part && (ldb & 15))) return NQ_ERR_ALIGNMENT;
+    if ((acc_out && (reinterpret_cast<uintptr_t>(acc_out) & 3)) || (Y && (reinterpret_cast<uintptr_t>(Y) & 1)))
+        return NQ_ERR_ALIGNMENT;
+    CUtensorMap tmA;
+    int st = encode_tensor_map_2d(&tmA, X, (uint64_t)K, (uint64_t)M, (uint64_t)ldx, kBK, kBM, true);
+    if (st != NQ_OK) return st;
+    return run_contraction(tmA, Bmat, ldb, part, n_bits, h_bits, w_scale, act_scale, bias, M, N, K, acc_out, ld_acc, Y,
+                           ldy, y_dtype, (cudaStream_t)stream);
+}
+
+}  // namespace
+}  // namespace nq
+
+extern "C" {
+
+int nq_gemm_full(const int8_t* X, int64_t ldx, const int8_t* W, int64_t ldw, const float* w_scale, float act_scale,
+                 const float* bias, int64_t M, int64_t N, int64_t K, int32_t* acc_out, int64_t ld_acc, void* Y,
+                 int64_t ldy, int y_dtype, void* stream) {
+    return nq::gemm_common(X, ldx, W, ldw, false, 8, 0, w_scale, act_scale, bias, M, N, K, acc_out, ld_acc, Y, ldy,
+                           y_dtype, stream);
+}
+
+int nq_gemm_part(const int8_t* X, int64_t ldx, const void* packed_high, int n_bits, int h_bits, const float* w_scale,
+                 float act_scale, const float* bias, int64_t M, int64_t N, int64_t K, int32_t* acc_out, int64_t ld_acc,
+                 void* Y, int64_t ldy, int y_dtype, void* stream) {
+    return nq::gemm_common(X, ldx, packed_high, 0, true, n_bits, h_bits, w_scale, act_scale, bias, M, N, K, acc_out,
+                           ld_acc, Y, ldy, y_dtype, stream);
+}
+
+}  // extern "C"
