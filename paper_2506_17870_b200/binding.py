@@ -9,13 +9,14 @@ raises ``NqLibraryError``.
 from __future__ import annotations
 
 import ctypes
+import os
 from pathlib import Path
 from typing import Optional, Sequence
 
 import torch
 
 _PKG = Path(__file__).resolve().parent
-_LIB_PATH = _PKG / "libnq_b200.so"
+_LIB_PATH = Path(os.environ.get("NQ_B200_LIB", _PKG / "libnq_b200.so"))   # override: a differently built copy
 _lib = None
 
 NQ_OK = 0

@@ -7,6 +7,11 @@
 // field of element 4q+i in its TOP k bits.  In that form every slice is a fixed bit range of every
 // byte, so moving between T and the slices is a mask, a shift and an OR per word -- four elements
 // per instruction -- and the nesting arithmetic (Eq. 5, 6, 10) is done on four bytes at a time.
+//
+// These kernels move 2-3 bytes per weight, so at HBM speed an SM has only a few integer
+// instructions per weight to spend.  For INT8 nesting (n = 8) every (h, compensate) pair therefore
+// gets its own instantiation with all shifts and masks as immediates; other n run a generic kernel
+// that takes them from registers.
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -20,15 +25,20 @@ namespace {
 constexpr uint32_t H4 = 0x80808080u;
 constexpr uint32_t L7 = 0x7f7f7f7fu;
 
-__device__ __forceinline__ uint32_t rep8(uint32_t b) { return (b & 0xffu) * 0x01010101u; }
+__host__ __device__ constexpr uint32_t rep8(uint32_t b) { return (b & 0xffu) * 0x01010101u; }
 
-// per-byte wrapping add / subtract, unsigned saturating subtract
-__device__ __forceinline__ uint32_t add4(uint32_t a, uint32_t b) {
-    return ((a & L7) + (b & L7)) ^ ((a ^ b) & H4);
-}
+// per-byte wrapping subtract
 __device__ __forceinline__ uint32_t sub4(uint32_t a, uint32_t b) {
     return ((a | H4) - (b & L7)) ^ ((a ^ ~b) & H4);
 }
+// per-byte unsigned saturating subtract for a subtrahend whose bytes are all below 0x80
+__device__ __forceinline__ uint32_t subsat_small_u4(uint32_t a, uint32_t s) {
+    uint32_t d = ((a | H4) - s) ^ (~a & H4);      // wrapping a - s
+    uint32_t under = ~a & d & H4;                 // top bit went 0 -> 1: the byte wrapped below zero
+    uint32_t kill = (under >> 7) * 0xffu;
+    return d & ~kill;
+}
+// the same for any subtrahend
 __device__ __forceinline__ uint32_t subsat_u4(uint32_t a, uint32_t b) {
     uint32_t d = sub4(a, b);
     uint32_t borrow = ((~a & b) | (~(a ^ b) & d)) & H4;   // borrow out of each byte
@@ -41,40 +51,87 @@ __device__ __forceinline__ uint32_t nonzero4(uint32_t x) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// nesting parameters: the same member names at run time (Nest) and at compile time (SNest)
+// ---------------------------------------------------------------------------------------------
+struct Nest {
+    int n, h, l, lb, comp;
+    uint32_t bias, mask_n, mask_h, mask_l, mask_lb, bit_l;
+    __device__ Nest(int n_, int h_, int comp_) : n(n_), h(h_), l(n_ - h_), lb(n_ - h_ + (comp_ ? 1 : 0)), comp(comp_) {
+        bias = rep8(1u << (n - 1));
+        mask_n = rep8((1u << n) - 1u);
+        mask_h = rep8((1u << h) - 1u);
+        mask_l = rep8((1u << l) - 1u);
+        mask_lb = rep8((1u << lb) - 1u);
+        bit_l = rep8(1u << l);
+    }
+};
+
+template <int N_, int H_, int COMP_>
+struct SNest {
+    static constexpr int n = N_, h = H_, l = N_ - H_, lb = N_ - H_ + (COMP_ ? 1 : 0), comp = COMP_;
+    static constexpr uint32_t bias = rep8(1u << (N_ - 1));
+    static constexpr uint32_t mask_n = rep8((1u << N_) - 1u);
+    static constexpr uint32_t mask_h = rep8((1u << H_) - 1u);
+    static constexpr uint32_t mask_l = rep8((1u << (N_ - H_)) - 1u);
+    static constexpr uint32_t mask_lb = rep8((1u << (N_ - H_ + (COMP_ ? 1 : 0))) - 1u);
+    static constexpr uint32_t bit_l = rep8(1u << (N_ - H_));
+    __device__ SNest(int, int, int) {}
+};
+
+// ---------------------------------------------------------------------------------------------
 // packed side: one unit <-> eight top-aligned words
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ void load_unit_top(const uint8_t* __restrict__ group, int unit, int bits,
-                                              uint32_t (&T)[8]) {
+struct PackedRaw {
+    uint4 a, b;      // 8-bit slice (two 16-byte halves) or, for narrower fields, a = the 4-bit slice
+    uint2 c;         // 2-bit slice
+    uint32_t d;      // 1-bit slice
+};
+
+__device__ __forceinline__ void load_packed_raw(const uint8_t* __restrict__ group, int unit, int bits, PackedRaw& r) {
     if (bits == 8) {
         const uint4* p = reinterpret_cast<const uint4*>(group + unit * 32);
-        uint4 a = __ldg(p), b = __ldg(p + 1);
-        T[0] = a.x; T[1] = a.y; T[2] = a.z; T[3] = a.w; T[4] = b.x; T[5] = b.y; T[6] = b.z; T[7] = b.w;
+        r.a = __ldg(p); r.b = __ldg(p + 1);
+        return;
+    }
+    int off = 0;
+    if (bits & 4) { r.a = __ldg(reinterpret_cast<const uint4*>(group + unit * 16)); off = 64; }
+    if (bits & 2) { r.c = __ldg(reinterpret_cast<const uint2*>(group + off + unit * 8)); off += 32; }
+    if (bits & 1) { r.d = __ldg(reinterpret_cast<const uint32_t*>(group + off + unit * 4)); }
+}
+
+__device__ __forceinline__ void expand_packed_raw(const PackedRaw& r, int bits, uint32_t (&T)[8]) {
+    if (bits == 8) {
+        T[0] = r.a.x; T[1] = r.a.y; T[2] = r.a.z; T[3] = r.a.w; T[4] = r.b.x; T[5] = r.b.y; T[6] = r.b.z; T[7] = r.b.w;
         return;
     }
 #pragma unroll
     for (int q = 0; q < 8; ++q) T[q] = 0;
-    int off = 0, used = 0;
+    int used = 0;
     if (bits & 4) {
-        uint4 w = __ldg(reinterpret_cast<const uint4*>(group + unit * 16));
-        T[0] = w.x & 0xf0f0f0f0u; T[1] = (w.x << 4) & 0xf0f0f0f0u;
-        T[2] = w.y & 0xf0f0f0f0u; T[3] = (w.y << 4) & 0xf0f0f0f0u;
-        T[4] = w.z & 0xf0f0f0f0u; T[5] = (w.z << 4) & 0xf0f0f0f0u;
-        T[6] = w.w & 0xf0f0f0f0u; T[7] = (w.w << 4) & 0xf0f0f0f0u;
-        off = 64; used = 4;
+        T[0] = r.a.x & 0xf0f0f0f0u; T[1] = (r.a.x << 4) & 0xf0f0f0f0u;
+        T[2] = r.a.y & 0xf0f0f0f0u; T[3] = (r.a.y << 4) & 0xf0f0f0f0u;
+        T[4] = r.a.z & 0xf0f0f0f0u; T[5] = (r.a.z << 4) & 0xf0f0f0f0u;
+        T[6] = r.a.w & 0xf0f0f0f0u; T[7] = (r.a.w << 4) & 0xf0f0f0f0u;
+        used = 4;
     }
+    // a narrower slice lands below the bits already placed: one net shift and one masked OR per word
     if (bits & 2) {
-        uint2 w = __ldg(reinterpret_cast<const uint2*>(group + off + unit * 8));
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
-            uint32_t word = (q < 4) ? w.x : w.y;
-            T[q] |= ((word << (2 * (q & 3))) & 0xc0c0c0c0u) >> used;
+            const uint32_t word = (q < 4) ? r.c.x : r.c.y;
+            const int net = 2 * (q & 3) - used;          // left shift if positive
+            const uint32_t moved = net >= 0 ? (word << net) : (word >> (-net));
+            T[q] |= moved & (0xc0c0c0c0u >> used);
         }
-        off += 32; used += 2;
+        used += 2;
     }
     if (bits & 1) {
-        uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(group + off + unit * 4));
 #pragma unroll
-        for (int q = 0; q < 8; ++q) T[q] |= ((w << q) & H4) >> used;
+        for (int q = 0; q < 8; ++q) {
+            const int net = q - used;
+            const uint32_t moved = net >= 0 ? (r.d << net) : (r.d >> (-net));
+            T[q] |= moved & (H4 >> used);
+        }
     }
 }
 
@@ -100,7 +157,9 @@ __device__ __forceinline__ void store_unit_top(uint8_t* __restrict__ group, int 
         uint2 w = make_uint2(0u, 0u);
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
-            uint32_t piece = ((T[q] << used) & 0xc0c0c0c0u) >> (2 * (q & 3));
+            const int net = used - 2 * (q & 3);          // left shift if positive
+            const uint32_t moved = net >= 0 ? (T[q] << net) : (T[q] >> (-net));
+            const uint32_t piece = moved & (0xc0c0c0c0u >> (2 * (q & 3)));
             if (q < 4) w.x |= piece; else w.y |= piece;
         }
         *reinterpret_cast<uint2*>(group + off + unit * 8) = w;
@@ -109,7 +168,11 @@ __device__ __forceinline__ void store_unit_top(uint8_t* __restrict__ group, int 
     if (bits & 1) {
         uint32_t w = 0;
 #pragma unroll
-        for (int q = 0; q < 8; ++q) w |= ((T[q] << used) & H4) >> q;
+        for (int q = 0; q < 8; ++q) {
+            const int net = used - q;
+            const uint32_t moved = net >= 0 ? (T[q] << net) : (T[q] >> (-net));
+            w |= moved & (H4 >> q);
+        }
         *reinterpret_cast<uint32_t*>(group + off + unit * 4) = w;
     }
 }
@@ -117,24 +180,38 @@ __device__ __forceinline__ void store_unit_top(uint8_t* __restrict__ group, int 
 // ---------------------------------------------------------------------------------------------
 // unpacked side: 32 int8 of one row <-> eight words, with a byte-wise path for ragged / unaligned rows
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ void load_unit_i8(const int8_t* __restrict__ row, int64_t c0, int64_t cols,
-                                             bool vec_ok, uint32_t (&V)[8]) {
-    if (vec_ok && c0 + 32 <= cols) {
-        const uint4* p = reinterpret_cast<const uint4*>(row + c0);
-        uint4 a = __ldg(p), b = __ldg(p + 1);
-        V[0] = a.x; V[1] = a.y; V[2] = a.z; V[3] = a.w; V[4] = b.x; V[5] = b.y; V[6] = b.z; V[7] = b.w;
-    } else {
+struct I8Raw {
+    uint4 a, b;
+    bool vec;        // loaded with vector loads; otherwise the byte-wise path runs at use time
+};
+
+__device__ __forceinline__ void load_unit_i8_bytes(const int8_t* __restrict__ row, int64_t c0, int64_t cols, uint32_t (&V)[8]) {
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            uint32_t w = 0;
+    for (int q = 0; q < 8; ++q) {
+        uint32_t w = 0;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                int64_t c = c0 + q * 4 + i;
-                uint32_t b = (c < cols) ? (uint32_t)(uint8_t)row[c] : 0u;
-                w |= b << (8 * i);
-            }
-            V[q] = w;
+        for (int i = 0; i < 4; ++i) {
+            int64_t c = c0 + q * 4 + i;
+            uint32_t b = (c < cols) ? (uint32_t)(uint8_t)row[c] : 0u;
+            w |= b << (8 * i);
         }
+        V[q] = w;
+    }
+}
+
+__device__ __forceinline__ void load_i8_raw(const int8_t* __restrict__ row, int64_t c0, int64_t cols, bool vec_ok, I8Raw& r) {
+    r.vec = vec_ok && c0 + 32 <= cols;
+    if (r.vec) {
+        const uint4* p = reinterpret_cast<const uint4*>(row + c0);
+        r.a = __ldg(p); r.b = __ldg(p + 1);
+    }
+}
+__device__ __forceinline__ void expand_i8_raw(const I8Raw& r, const int8_t* __restrict__ row, int64_t c0, int64_t cols,
+                                              uint32_t (&V)[8]) {
+    if (r.vec) {
+        V[0] = r.a.x; V[1] = r.a.y; V[2] = r.a.z; V[3] = r.a.w; V[4] = r.b.x; V[5] = r.b.y; V[6] = r.b.z; V[7] = r.b.w;
+    } else {
+        load_unit_i8_bytes(row, c0, cols, V);
     }
 }
 
@@ -159,28 +236,17 @@ __device__ __forceinline__ void store_unit_i8(int8_t* __restrict__ row, int64_t 
 // the nesting arithmetic on four bytes at a time.  "Biased" means value + 2^(n-1), an unsigned
 // n-bit number; in that domain w_high + 2^(h-1) is simply the top h bits.
 // ---------------------------------------------------------------------------------------------
-struct Nest {
-    int n, h, l, lb, comp;
-    uint32_t bias, mask_n, mask_h, mask_l, mask_lb, bit_l;
-    __device__ Nest(int n_, int h_, int comp_) : n(n_), h(h_), l(n_ - h_), lb(n_ - h_ + (comp_ ? 1 : 0)), comp(comp_) {
-        bias = rep8(1u << (n - 1));
-        mask_n = rep8((1u << n) - 1u);
-        mask_h = rep8((1u << h) - 1u);
-        mask_l = rep8((1u << l) - 1u);
-        mask_lb = rep8((1u << lb) - 1u);
-        bit_l = rep8(1u << l);
-    }
-};
 
 // Eq. 6 with the mask-given rounding, then Eq. 10 / compensation.  V, M: int8 weights and mask bytes.
-__device__ __forceinline__ void decompose_word(const Nest& N, uint32_t V, uint32_t M, uint32_t& Thi, uint32_t& Tlo) {
+template <class NestT>
+__device__ __forceinline__ void decompose_word(const NestT& N, uint32_t V, uint32_t M, uint32_t& Thi, uint32_t& Tlo) {
     uint32_t wu = (V ^ N.bias) & N.mask_n;                 // w + 2^(n-1)
     uint32_t down = (wu >> N.l) & N.mask_h;                // floor(w / 2^l) + 2^(h-1)
-    uint32_t rem = wu & N.mask_l;
-    uint32_t up = nonzero4(rem) & nonzero4(M);             // round up only off a multiple of 2^l
+    uint32_t rem_nz = ((wu & N.mask_l) + L7) & H4;         // remainder != 0 (it is below 0x80: the add stays in its byte)
+    uint32_t up = (rem_nz >> 7) & nonzero4(M);             // round up only off a multiple of 2^l
     uint32_t whb = down + up;                              // <= 2^h per byte: no carry between bytes
     whb -= (whb >> N.h) & 0x01010101u;                     // clip to 2^h - 1 (max_high, biased)
-    Thi = ((whb ^ rep8(1u << (N.h - 1))) & N.mask_h) << (8 - N.h);
+    Thi = (whb << (8 - N.h)) ^ H4;                         // two's complement again, field in the top h bits
     // w_low = w - w_high * 2^l; modulo 2^(l+1) that is the low l bits of w plus one borrow bit
     uint32_t lo = (wu ^ (whb << N.l)) & rep8((2u << N.l) - 1u);
     if (!N.comp) {
@@ -194,7 +260,8 @@ __device__ __forceinline__ void decompose_word(const Nest& N, uint32_t V, uint32
 }
 
 // Eq. 5: shift, add the signed low field, clip to INTn.  Returns int8 bytes.
-__device__ __forceinline__ uint32_t recompose_word(const Nest& N, uint32_t Thi, uint32_t Tlo) {
+template <class NestT>
+__device__ __forceinline__ uint32_t recompose_word(const NestT& N, uint32_t Thi, uint32_t Tlo) {
     uint32_t x = ((Thi >> (8 - N.n)) & N.mask_n) ^ N.bias;     // (w_high + 2^(h-1)) << l
     uint32_t lo = (Tlo >> (8 - N.lb)) & N.mask_lb;
     uint32_t a, s;
@@ -206,12 +273,14 @@ __device__ __forceinline__ uint32_t recompose_word(const Nest& N, uint32_t Thi, 
         a = x | (lo ^ half);
         s = half;
     }
-    uint32_t wu = subsat_u4(a, s);                              // the only clip that can bind is the lower one
+    // the only clip that can bind is the lower one (result below -2^(n-1)): an unsigned saturating subtract
+    uint32_t wu = (N.comp && N.l == 7) ? subsat_u4(a, s) : subsat_small_u4(a, s);
     return sub4(wu, N.bias);
 }
 
 // (w_int - w_low) / 2^l as an h-bit field
-__device__ __forceinline__ uint32_t drop_low_word(const Nest& N, uint32_t V, uint32_t Tlo) {
+template <class NestT>
+__device__ __forceinline__ uint32_t drop_low_word(const NestT& N, uint32_t V, uint32_t Tlo) {
     uint32_t lo = (Tlo >> (8 - N.lb)) & N.mask_lb;
     uint32_t m = rep8(1u << (N.lb - 1));
     uint32_t lo_signed = sub4(lo ^ m, m);
@@ -242,61 +311,71 @@ struct TensorView {
 
 enum Op { OP_DECOMPOSE = 0, OP_RECOMPOSE = 1, OP_DROP_LOW = 2, OP_UNPACK = 3, OP_PACK = 4 };
 
-template <int OP>
-__device__ __forceinline__ void do_unit(const TensorView& t, int64_t unit_index, const Nest& N, int bits) {
-    const int64_t units_per_row = ((t.cols + 127) / 128) * 4;
-    const int64_t row = unit_index / units_per_row;
-    const int64_t ur = unit_index - row * units_per_row;
-    const int64_t group = ur >> 2;
+template <int OP, class NestT>
+__device__ __forceinline__ void do_unit(const TensorView& t, int64_t unit_index, const NestT& N, int bits) {
+    const int64_t units_per_row = ((t.cols + 127) >> 7) << 2;
+    int64_t row, ur;
+    if (((unit_index | units_per_row) >> 32) == 0) {          // the usual case: 32-bit divide
+        const uint32_t r32 = (uint32_t)unit_index / (uint32_t)units_per_row;
+        row = r32;
+        ur = (uint32_t)unit_index - r32 * (uint32_t)units_per_row;
+    } else {
+        row = unit_index / units_per_row;
+        ur = unit_index - row * units_per_row;
+    }
+    const int64_t group = row * (units_per_row >> 2) + (ur >> 2);
     const int unit = (int)(ur & 3);
     const int64_t c0 = ur * 32;
     const bool vec_ok = ((t.ld & 15) == 0) && ((reinterpret_cast<uintptr_t>(t.w) & 15) == 0) &&
                         (OP != OP_DECOMPOSE || (reinterpret_cast<uintptr_t>(t.mask) & 15) == 0);
     int8_t* wrow = t.w + row * t.ld;
     uint32_t A[8], Bv[8];
+    PackedRaw p0, p1;
+    I8Raw v0, v1;
     if (OP == OP_DECOMPOSE) {
-        uint8_t* ghi = t.hi + (row * (units_per_row >> 2) + group) * 16 * N.h;
-        uint8_t* glo = t.lo + (row * (units_per_row >> 2) + group) * 16 * N.lb;
-        load_unit_i8(wrow, c0, t.cols, vec_ok, A);
-        load_unit_i8(reinterpret_cast<const int8_t*>(t.mask) + row * t.ld, c0, t.cols, vec_ok, Bv);
+        const int8_t* mrow = reinterpret_cast<const int8_t*>(t.mask) + row * t.ld;
+        load_i8_raw(wrow, c0, t.cols, vec_ok, v0);
+        load_i8_raw(mrow, c0, t.cols, vec_ok, v1);
+        expand_i8_raw(v0, wrow, c0, t.cols, A);
+        expand_i8_raw(v1, mrow, c0, t.cols, Bv);
 #pragma unroll
         for (int q = 0; q < 8; ++q) decompose_word(N, A[q], Bv[q], A[q], Bv[q]);
-        store_unit_top(ghi, unit, N.h, A);
-        store_unit_top(glo, unit, N.lb, Bv);
+        store_unit_top(t.hi + group * 16 * N.h, unit, N.h, A);
+        store_unit_top(t.lo + group * 16 * N.lb, unit, N.lb, Bv);
     } else if (OP == OP_RECOMPOSE) {
-        const uint8_t* ghi = t.hi + (row * (units_per_row >> 2) + group) * 16 * N.h;
-        const uint8_t* glo = t.lo + (row * (units_per_row >> 2) + group) * 16 * N.lb;
-        load_unit_top(ghi, unit, N.h, A);
-        load_unit_top(glo, unit, N.lb, Bv);
+        load_packed_raw(t.hi + group * 16 * N.h, unit, N.h, p0);
+        load_packed_raw(t.lo + group * 16 * N.lb, unit, N.lb, p1);
+        expand_packed_raw(p0, N.h, A);
+        expand_packed_raw(p1, N.lb, Bv);
 #pragma unroll
         for (int q = 0; q < 8; ++q) A[q] = recompose_word(N, A[q], Bv[q]);
         store_unit_i8(wrow, c0, t.cols, vec_ok, A);
     } else if (OP == OP_DROP_LOW) {
-        uint8_t* ghi = t.hi + (row * (units_per_row >> 2) + group) * 16 * N.h;
-        const uint8_t* glo = t.lo + (row * (units_per_row >> 2) + group) * 16 * N.lb;
-        load_unit_i8(wrow, c0, t.cols, vec_ok, A);
-        load_unit_top(glo, unit, N.lb, Bv);
+        load_i8_raw(wrow, c0, t.cols, vec_ok, v0);
+        load_packed_raw(t.lo + group * 16 * N.lb, unit, N.lb, p1);
+        expand_i8_raw(v0, wrow, c0, t.cols, A);
+        expand_packed_raw(p1, N.lb, Bv);
 #pragma unroll
         for (int q = 0; q < 8; ++q) A[q] = drop_low_word(N, A[q], Bv[q]);
-        store_unit_top(ghi, unit, N.h, A);
+        store_unit_top(t.hi + group * 16 * N.h, unit, N.h, A);
     } else if (OP == OP_UNPACK) {
-        const uint8_t* g = t.hi + (row * (units_per_row >> 2) + group) * 16 * bits;
-        load_unit_top(g, unit, bits, A);
+        load_packed_raw(t.hi + group * 16 * bits, unit, bits, p0);
+        expand_packed_raw(p0, bits, A);
 #pragma unroll
         for (int q = 0; q < 8; ++q) A[q] = top_to_values(A[q], bits);
         store_unit_i8(wrow, c0, t.cols, vec_ok, A);
     } else {
-        uint8_t* g = t.hi + (row * (units_per_row >> 2) + group) * 16 * bits;
-        load_unit_i8(wrow, c0, t.cols, vec_ok, A);
+        load_i8_raw(wrow, c0, t.cols, vec_ok, v0);
+        expand_i8_raw(v0, wrow, c0, t.cols, A);
 #pragma unroll
         for (int q = 0; q < 8; ++q) A[q] = values_to_top(A[q], bits);
-        store_unit_top(g, unit, bits, A);
+        store_unit_top(t.hi + group * 16 * bits, unit, bits, A);
     }
 }
 
-template <int OP>
-__global__ void __launch_bounds__(256) codec_kernel(TensorView t, int64_t total_units, int n, int h, int comp, int bits) {
-    const Nest N(n, h, comp);
+template <int OP, class NestT>
+__global__ void __launch_bounds__(256, 4) codec_kernel(TensorView t, int64_t total_units, int n, int h, int comp, int bits) {
+    const NestT N(n, h, comp);
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < total_units; u += stride)
         do_unit<OP>(t, u, N, bits);
@@ -313,10 +392,10 @@ struct BatchEntry {
 };
 static_assert(sizeof(BatchEntry) == 64, "table entry is 64 bytes");
 
-template <int OP>
-__global__ void __launch_bounds__(256) codec_batched_kernel(const BatchEntry* __restrict__ table, int count,
-                                                            int64_t total_units, int n, int h, int comp) {
-    const Nest N(n, h, comp);
+template <int OP, class NestT>
+__global__ void __launch_bounds__(256, 4) codec_batched_kernel(const BatchEntry* __restrict__ table, int count,
+                                                               int64_t total_units, int n, int h, int comp) {
+    const NestT N(n, h, comp);
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < total_units; u += stride) {
         int lo = 0, hi = count - 1;                 // last entry whose first_unit <= u
@@ -341,11 +420,52 @@ inline int launch_blocks(int64_t total_units) {
 inline bool nest_ok(int n, int h) { return n >= 2 && n <= 8 && h >= 1 && h < n; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
+// launchers: INT8 nesting gets the compile-time instantiation of its (h, compensate)
+template <int OP, class NestT>
+void launch_one(const TensorView& t, int64_t total, int n, int h, int comp, int bits, cudaStream_t s) {
+    codec_kernel<OP, NestT><<<launch_blocks(total), 256, 0, s>>>(t, total, n, h, comp, bits);
+}
+template <int OP, class NestT>
+void launch_batch(const BatchEntry* table, int count, int64_t total, int n, int h, int comp, cudaStream_t s) {
+    codec_batched_kernel<OP, NestT><<<launch_blocks(total), 256, 0, s>>>(table, count, total, n, h, comp);
+}
+
+template <int OP, int H>
+void dispatch_comp(bool batched, const TensorView& t, const BatchEntry* table, int count, int64_t total, int comp,
+                   cudaStream_t s) {
+    if (comp) {
+        if (batched) launch_batch<OP, SNest<8, H, 1>>(table, count, total, 8, H, 1, s);
+        else launch_one<OP, SNest<8, H, 1>>(t, total, 8, H, 1, 0, s);
+    } else {
+        if (batched) launch_batch<OP, SNest<8, H, 0>>(table, count, total, 8, H, 0, s);
+        else launch_one<OP, SNest<8, H, 0>>(t, total, 8, H, 0, 0, s);
+    }
+}
+
+template <int OP>
+void dispatch_nest(bool batched, const TensorView& t, const BatchEntry* table, int count, int64_t total, int n, int h,
+                   int comp, cudaStream_t s) {
+    if (n == 8) {
+        switch (h) {
+            case 1: return dispatch_comp<OP, 1>(batched, t, table, count, total, comp, s);
+            case 2: return dispatch_comp<OP, 2>(batched, t, table, count, total, comp, s);
+            case 3: return dispatch_comp<OP, 3>(batched, t, table, count, total, comp, s);
+            case 4: return dispatch_comp<OP, 4>(batched, t, table, count, total, comp, s);
+            case 5: return dispatch_comp<OP, 5>(batched, t, table, count, total, comp, s);
+            case 6: return dispatch_comp<OP, 6>(batched, t, table, count, total, comp, s);
+            default: return dispatch_comp<OP, 7>(batched, t, table, count, total, comp, s);
+        }
+    }
+    if (batched) launch_batch<OP, Nest>(table, count, total, n, h, comp, s);
+    else launch_one<OP, Nest>(t, total, n, h, comp, 0, s);
+}
+
 template <int OP>
 int run_single(TensorView t, int n, int h, int comp, int bits, void* stream) {
     if (t.rows == 0 || t.cols == 0) return NQ_OK;
     int64_t total = t.rows * ((t.cols + 127) / 128) * 4;
-    codec_kernel<OP><<<launch_blocks(total), 256, 0, (cudaStream_t)stream>>>(t, total, n, h, comp, bits);
+    if (OP == OP_UNPACK || OP == OP_PACK) launch_one<OP, Nest>(t, total, n, h, comp, bits, (cudaStream_t)stream);
+    else dispatch_nest<OP>(false, t, nullptr, 0, total, n, h, comp, (cudaStream_t)stream);
     return cudaGetLastError() == cudaSuccess ? NQ_OK : NQ_ERR_CUDA;
 }
 
@@ -461,11 +581,9 @@ static int run_batched(int op, const void* table, int count, int64_t units, int 
     if (!nest_ok(n, h)) return NQ_ERR_UNSUPPORTED;
     if (count == 0 || units == 0) return NQ_OK;
     const BatchEntry* entries = reinterpret_cast<const BatchEntry*>(table);
-    int blocks = launch_blocks(units);
-    if (op == OP_RECOMPOSE)
-        codec_batched_kernel<OP_RECOMPOSE><<<blocks, 256, 0, (cudaStream_t)stream>>>(entries, count, units, n, h, comp);
-    else
-        codec_batched_kernel<OP_DROP_LOW><<<blocks, 256, 0, (cudaStream_t)stream>>>(entries, count, units, n, h, comp);
+    TensorView none{};
+    if (op == OP_RECOMPOSE) dispatch_nest<OP_RECOMPOSE>(true, none, entries, count, units, n, h, comp, (cudaStream_t)stream);
+    else dispatch_nest<OP_DROP_LOW>(true, none, entries, count, units, n, h, comp, (cudaStream_t)stream);
     return cudaGetLastError() == cudaSuccess ? NQ_OK : NQ_ERR_CUDA;
 }
 
