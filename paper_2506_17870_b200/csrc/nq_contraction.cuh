@@ -30,7 +30,23 @@ constexpr int kStagesPart = 3;
 constexpr int kPackedStages = 2;
 constexpr int kGroupM = 16;        // tile rasterisation: 16 M-tiles share a band of N-tiles
 
+// How the A operand is gathered.
+//   kModeGemm    A is a plain [M, K] matrix: one 2-D tile per stage.
+//   kModeConv128 implicit GEMM, Cin a multiple of 128: a stage is 128 channels of ONE filter tap for a
+//                tw x th x tb rectangle of output pixels, fetched by one 4-D tile load from the NHWC tensor.
+//   kModeConv64  implicit GEMM, Cin = 64: a stage is TWO taps x 64 channels, held as two sub-tiles of
+//                64-byte rows (64-byte swizzle) for A and for B alike.
+constexpr int kModeGemm = 0, kModeConv128 = 1, kModeConv64 = 2;
+
+struct ConvGeom {
+    int B, Ho, Wo, S, taps, stride, pad;
+    int cblocks;                     // kModeConv128: Cin / 128
+    int tw_log2, th_log2;            // tile = 2^tw x 2^th output pixels of 128 / (2^tw * 2^th) images
+    int tiles_w, tiles_h;
+};
+
 struct ContractionArgs {
+    ConvGeom g;
     int M, N, K;
     int m_tiles, n_tiles, k_blocks;
     const float* w_scale;
@@ -100,7 +116,20 @@ __device__ __forceinline__ void unpack_unit_top(const uint8_t* group, int unit, 
     }
 }
 
-template <int BN, bool PART>
+struct TileOrigin {      // where an M-tile starts, in output-pixel coordinates (convolution modes)
+    int b0, p0, q0;
+};
+__device__ __forceinline__ TileOrigin conv_tile_origin(const ConvGeom& g, int mt) {
+    TileOrigin o;
+    const int qt = mt % g.tiles_w;
+    const int rest = mt / g.tiles_w;
+    o.q0 = qt << g.tw_log2;
+    o.p0 = (rest % g.tiles_h) << g.th_log2;
+    o.b0 = (rest / g.tiles_h) << (7 - g.tw_log2 - g.th_log2);
+    return o;
+}
+
+template <int BN, bool PART, int MODE>
 __global__ void __launch_bounds__(PART ? 320 : 192, 1)
 contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                    const ContractionArgs p) {
@@ -173,18 +202,35 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                     const uint32_t s = it % STAGES, use = it / STAGES;
                     if (!(ok = mbar_wait(smem_u32(&empty[s]), (use & 1) ^ 1, abort_flag, p.status, 0x10u))) break;
                     const uint32_t fb = smem_u32(&full[s]);
-                    if (PART) {
-                        mbar_arrive_expect_tx(fb, A_BYTES);
+                    // bytes this stage brings in: A always; B too in full-bit mode
+                    int n_sub = 1;                                       // kModeConv64: taps present in this stage
+                    if (MODE == kModeConv64) n_sub = min(2, p.g.taps - 2 * kb);
+                    const uint32_t a_bytes = (MODE == kModeConv64) ? n_sub * (A_BYTES / 2) : A_BYTES;
+                    const uint32_t b_bytes = PART ? 0u : ((MODE == kModeConv64) ? n_sub * (B_BYTES / 2) : B_BYTES);
+                    mbar_arrive_expect_tx(fb, a_bytes + b_bytes);
+                    if (MODE == kModeGemm) {
                         tma_load_2d(smem_u32(sA + s * A_BYTES), &tmA, kb * kBK, mt * kBM, fb);
+                    } else {
+                        const TileOrigin o = conv_tile_origin(p.g, mt);
+                        for (int sub = 0; sub < n_sub; ++sub) {
+                            const int tap = (MODE == kModeConv64) ? 2 * kb + sub : kb / p.g.cblocks;
+                            const int c0 = (MODE == kModeConv64) ? 0 : (kb % p.g.cblocks) * 128;
+                            const int r = tap / p.g.S, sx = tap - r * p.g.S;
+                            tma_load_4d(smem_u32(sA + s * A_BYTES + sub * (A_BYTES / 2)), &tmA, c0,
+                                        o.q0 * p.g.stride - p.g.pad + sx, o.p0 * p.g.stride - p.g.pad + r, o.b0, fb);
+                        }
+                    }
+                    if (PART) {
                         const uint32_t ps = pit % kPackedStages, puse = pit / kPackedStages;
                         if (!(ok = mbar_wait(smem_u32(&pempty[ps]), (puse & 1) ^ 1, abort_flag, p.status, 0x11u))) break;
                         const uint32_t pb = smem_u32(&pfull[ps]);
                         mbar_arrive_expect_tx(pb, packed_bytes);
                         tma_load_2d(smem_u32(sP + ps * packed_bytes), &tmB, kb * 16 * p.h_bits, nt * BN, pb);
                         ++pit;
+                    } else if (MODE == kModeConv64) {
+                        for (int sub = 0; sub < n_sub; ++sub)
+                            tma_load_2d(smem_u32(sB + s * B_BYTES + sub * (B_BYTES / 2)), &tmB, kb * kBK + sub * 64, nt * BN, fb);
                     } else {
-                        mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
-                        tma_load_2d(smem_u32(sA + s * A_BYTES), &tmA, kb * kBK, mt * kBM, fb);
                         tma_load_2d(smem_u32(sB + s * B_BYTES), &tmB, kb * kBK, nt * BN, fb);
                     }
                 }
@@ -209,11 +255,22 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                     const uint32_t s = it % STAGES, use = it / STAGES;
                     if (!(ok = mbar_wait(smem_u32(&full[s]), use & 1, abort_flag, p.status, 0x21u))) break;
                     tc_fence_after_sync();
-                    const uint64_t da = smem_desc_sw128(smem_u32(sA + s * A_BYTES));
-                    const uint64_t db = smem_desc_sw128(smem_u32(sB + s * B_BYTES));
+                    if (MODE == kModeConv64) {
+                        const int n_sub = min(2, p.g.taps - 2 * kb);
+                        for (int sub = 0; sub < n_sub; ++sub) {
+                            const uint64_t da = smem_desc_sw64(smem_u32(sA + s * A_BYTES + sub * (A_BYTES / 2)));
+                            const uint64_t db = smem_desc_sw64(smem_u32(sB + s * B_BYTES + sub * (B_BYTES / 2)));
 #pragma unroll
-                    for (int k = 0; k < kBK / 32; ++k)   // 32 bytes of K per instruction: +2 in the address field
-                        mma_i8(d_tmem, da + 2 * k, db + 2 * k, IDESC, (kb | k) != 0);
+                            for (int k = 0; k < 2; ++k)
+                                mma_i8(d_tmem, da + 2 * k, db + 2 * k, IDESC, (kb | sub | k) != 0);
+                        }
+                    } else {
+                        const uint64_t da = smem_desc_sw128(smem_u32(sA + s * A_BYTES));
+                        const uint64_t db = smem_desc_sw128(smem_u32(sB + s * B_BYTES));
+#pragma unroll
+                        for (int k = 0; k < kBK / 32; ++k)   // 32 bytes of K per instruction: +2 in the address field
+                            mma_i8(d_tmem, da + 2 * k, db + 2 * k, IDESC, (kb | k) != 0);
+                    }
                     mma_commit(smem_u32(&empty[s]));       // stage reusable once these MMAs have read it
                 }
                 if (ok) mma_commit(smem_u32(&tfull[buf]));   // accumulator complete
@@ -255,8 +312,21 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after_sync();
-            const long long row = (long long)mt * kBM + quarter * 32 + lane;
-            const bool row_ok = row < p.M;
+            long long row;
+            bool row_ok;
+            if (MODE == kModeGemm) {
+                row = (long long)mt * kBM + quarter * 32 + lane;
+                row_ok = row < p.M;
+            } else {
+                // tile row -> output pixel: the low bits walk the width, then the height, then the images
+                const TileOrigin o = conv_tile_origin(p.g, mt);
+                const int ml = quarter * 32 + lane;
+                const int qq = o.q0 + (ml & ((1 << p.g.tw_log2) - 1));
+                const int pp = o.p0 + ((ml >> p.g.tw_log2) & ((1 << p.g.th_log2) - 1));
+                const int bb = o.b0 + (ml >> (p.g.tw_log2 + p.g.th_log2));
+                row_ok = qq < p.g.Wo && pp < p.g.Ho && bb < p.g.B;
+                row = ((long long)bb * p.g.Ho + pp) * p.g.Wo + qq;
+            }
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t r[32];
@@ -348,10 +418,18 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                     const int row = task >> 2, unit = task & 3;
                     uint32_t T[8];
                     unpack_unit_top(src + row * 16 * h, unit, h, T);
-                    uint8_t* drow = dst + row * 128;
-                    const int sw = row & 7;
-                    *reinterpret_cast<uint4*>(drow + (((2 * unit) ^ sw) << 4)) = make_uint4(T[0], T[1], T[2], T[3]);
-                    *reinterpret_cast<uint4*>(drow + (((2 * unit + 1) ^ sw) << 4)) = make_uint4(T[4], T[5], T[6], T[7]);
+                    if (MODE == kModeConv64) {
+                        // two sub-tiles of 64-byte rows: units 0,1 feed the first, 2,3 the second; 64-byte swizzle
+                        uint8_t* drow = dst + (unit >> 1) * (B_BYTES / 2) + row * 64;
+                        const int sw = (row >> 1) & 3, c = (unit & 1) * 2;
+                        *reinterpret_cast<uint4*>(drow + ((c ^ sw) << 4)) = make_uint4(T[0], T[1], T[2], T[3]);
+                        *reinterpret_cast<uint4*>(drow + (((c + 1) ^ sw) << 4)) = make_uint4(T[4], T[5], T[6], T[7]);
+                    } else {
+                        uint8_t* drow = dst + row * 128;
+                        const int sw = row & 7;
+                        *reinterpret_cast<uint4*>(drow + (((2 * unit) ^ sw) << 4)) = make_uint4(T[0], T[1], T[2], T[3]);
+                        *reinterpret_cast<uint4*>(drow + (((2 * unit + 1) ^ sw) << 4)) = make_uint4(T[4], T[5], T[6], T[7]);
+                    }
                 }
                 fence_proxy_async_smem();              // these writes feed tcgen05.mma (async proxy)
                 __syncwarp();
@@ -371,5 +449,12 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         tmem_dealloc(tmem_base, TMEM_COLS);
     }
 }
+
+// Host launcher (defined with the GEMM entry points).  The A operand is reached through tmA: a plain 2-D map
+// of an [M, K] matrix (kModeGemm, geom == nullptr) or a 4-D map of NHWC activations (convolution modes).
+int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int m_tiles, int k_blocks,
+                    const void* Bmat, int64_t ldb, bool part, int n_bits, int h_bits,
+                    const float* w_scale, float act_scale, const float* bias, int64_t M, int64_t N, int64_t K,
+                    int32_t* acc_out, int64_t ld_acc, void* Y, int64_t ldy, int y_dtype, cudaStream_t stream);
 
 }  // namespace nq

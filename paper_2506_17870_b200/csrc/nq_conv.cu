@@ -1,19 +1,189 @@
-// Implicit-GEMM convolution entry points (under construction: the contraction core is shared with the GEMM).
+// Implicit-GEMM convolution on the nested weights: layout pre-passes, tile geometry, launch.
+//
+// The contraction itself is the kernel of nq_contraction.cuh.  Here the activations are brought to the
+// form its TMA producer reads:
+//   - Cin = 64 or a multiple of 128 (every ResNet layer but the stem): NHWC activations are read in place,
+//     one rectangle of output pixels and one filter tap at a time, by 4-D tile loads whose out-of-image
+//     coordinates return zeros (the zero padding).  NCHW input is first transposed into the workspace.
+//   - any other Cin (the 3-channel stem): the [M, K] patch matrix is written out explicitly into the
+//     workspace and the plain GEMM path runs on it.
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
 #include "../../include/nq.h"
+#include "nq_contraction.cuh"
+#include "nq_internal.cuh"
+
+namespace nq {
+namespace {
+
+// [B, C, HW] int8 -> [B, HW, C]; a block moves 64 channels x 64 pixels through shared memory
+__global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(const int8_t* __restrict__ in, int8_t* __restrict__ out,
+                                                           int C, int HW) {
+    __shared__ __align__(16) uint8_t tile[64][80];            // [pixel][channel], pitch 80 keeps rows 16-byte aligned
+    const int b = blockIdx.z, c0 = blockIdx.y * 64, p0 = blockIdx.x * 64;
+    const int8_t* src = in + ((size_t)b * C + c0) * HW;
+    int8_t* dst = out + (size_t)b * HW * C;
+    const int t = threadIdx.x;
+    const bool words = ((HW & 3) == 0) && ((reinterpret_cast<uintptr_t>(in) & 3) == 0);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int c = (t >> 4) + 16 * i, x4 = (t & 15) * 4;
+        uint32_t w = 0;
+        if (c0 + c < C) {
+            if (words && p0 + x4 + 3 < HW) {
+                w = *reinterpret_cast<const uint32_t*>(src + (size_t)c * HW + p0 + x4);
+            } else {
+                for (int j = 0; j < 4; ++j)
+                    if (p0 + x4 + j < HW) w |= (uint32_t)(uint8_t)src[(size_t)c * HW + p0 + x4 + j] << (8 * j);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) tile[x4 + j][c] = (uint8_t)(w >> (8 * j));
+    }
+    __syncthreads();
+    const int pix = t >> 2, cq = (t & 3) * 16;
+    if (p0 + pix < HW) {
+        if (c0 + cq + 16 <= C && (C & 15) == 0) {
+            *reinterpret_cast<uint4*>(dst + (size_t)(p0 + pix) * C + c0 + cq) = *reinterpret_cast<const uint4*>(&tile[pix][cq]);
+        } else {
+            for (int j = 0; j < 16; ++j)
+                if (c0 + cq + j < C) dst[(size_t)(p0 + pix) * C + c0 + cq + j] = (int8_t)tile[pix][cq + j];
+        }
+    }
+}
+
+// explicit patch matrix A[m, k], k = (r*S + s)*Cin + ci, row pitch ld (a multiple of 16), zero beyond K
+__global__ void __launch_bounds__(256) im2col_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ a, nq_conv_desc d,
+                                                     int Ho, int Wo, int K, int ld, long long chunks_total) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= chunks_total) return;
+    const int chunks_per_row = ld / 16;
+    const long long m = idx / chunks_per_row;
+    const int k0 = (int)(idx - m * chunks_per_row) * 16;
+    const int q = (int)(m % Wo);
+    const long long t = m / Wo;
+    const int p = (int)(t % Ho), b = (int)(t / Ho);
+    uint32_t w[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const int k = k0 + j;
+        uint32_t v = 0;
+        if (k < K) {
+            const int tap = k / d.Cin, ci = k - tap * d.Cin;
+            const int r = tap / d.S, s = tap - r * d.S;
+            const int ih = p * d.stride - d.pad + r, iw = q * d.stride - d.pad + s;
+            if (ih >= 0 && ih < d.H && iw >= 0 && iw < d.W) {
+                const size_t off = d.x_nchw ? (((size_t)b * d.Cin + ci) * d.H + ih) * d.W + iw
+                                            : (((size_t)b * d.H + ih) * d.W + iw) * d.Cin + ci;
+                v = (uint8_t)x[off];
+            }
+        }
+        w[j >> 2] |= v << (8 * (j & 3));
+    }
+    *reinterpret_cast<uint4*>(a + m * ld + k0) = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+bool implicit_ok(const nq_conv_desc& d) { return d.Cin == 64 || (d.Cin > 0 && d.Cin % 128 == 0); }
+
+bool desc_ok(const nq_conv_desc* d) {
+    return d && d->B > 0 && d->Cin > 0 && d->H > 0 && d->W > 0 && d->Cout > 0 && d->R > 0 && d->S > 0 && d->stride > 0 &&
+           d->pad >= 0 && d->H + 2 * d->pad >= d->R && d->W + 2 * d->pad >= d->S;
+}
+
+int out_dim(int in, int k, int stride, int pad) { return (in + 2 * pad - k) / stride + 1; }
+
+// rectangle of 2^tw x 2^th output pixels of 128 / 2^(tw+th) images that wastes the fewest tile rows
+void choose_tile(int B, int Ho, int Wo, int& tw_log2, int& th_log2) {
+    double best = 1e300;
+    tw_log2 = 3; th_log2 = 3;
+    for (int a = 7; a >= 0; --a)
+        for (int b = 7 - a; b >= 0; --b) {
+            const long long tw = 1 << a, th = 1 << b, tb = 128 >> (a + b);
+            const double cover = (double)((Wo + tw - 1) / tw * tw) * ((Ho + th - 1) / th * th) * ((B + tb - 1) / tb * tb);
+            if (cover < best) { best = cover; tw_log2 = a; th_log2 = b; }
+        }
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+}  // namespace
+}  // namespace nq
 
 extern "C" {
 
-int64_t nq_conv_workspace_bytes(const nq_conv_desc* desc) {
-    if (!desc) return -1;
-    return 0;
+int64_t nq_conv_workspace_bytes(const nq_conv_desc* d) {
+    if (!nq::desc_ok(d)) return -1;
+    if (nq::implicit_ok(*d)) return d->x_nchw ? (int64_t)d->B * d->H * d->W * d->Cin : 0;
+    const int64_t Ho = nq::out_dim(d->H, d->R, d->stride, d->pad), Wo = nq::out_dim(d->W, d->S, d->stride, d->pad);
+    const int64_t K = (int64_t)d->R * d->S * d->Cin;
+    return (int64_t)d->B * Ho * Wo * ((K + 15) / 16 * 16);
 }
 
-int nq_conv_implicit_gemm(const int8_t*, const void*, int64_t, int, int, int, const nq_conv_desc*, const float*, float,
-                          const float*, int32_t*, void*, int, void*, int64_t, void*) {
-    return NQ_ERR_UNSUPPORTED;
+int nq_conv_implicit_gemm(const int8_t* X, const void* Wt, int64_t ldw, int part_bit, int n_bits, int h_bits,
+                          const nq_conv_desc* d, const float* w_scale, float act_scale, const float* bias,
+                          int32_t* acc_out, void* Y, int y_dtype, void* workspace, int64_t workspace_bytes, void* stream_) {
+    using namespace nq;
+    if (!desc_ok(d)) return NQ_ERR_INVALID_ARG;
+    if (y_dtype != NQ_F32 && y_dtype != NQ_BF16) return NQ_ERR_INVALID_ARG;
+    if (part_bit && (n_bits < 2 || n_bits > 8 || h_bits < 1 || h_bits >= n_bits)) return NQ_ERR_UNSUPPORTED;
+    if (!X || !Wt || (!acc_out && !Y) || (Y && !w_scale)) return NQ_ERR_INVALID_ARG;
+    const int Ho = out_dim(d->H, d->R, d->stride, d->pad), Wo = out_dim(d->W, d->S, d->stride, d->pad);
+    const int64_t M = (int64_t)d->B * Ho * Wo, N = d->Cout, K = (int64_t)d->R * d->S * d->Cin;
+    if (K >= (1 << 17) || M > (1ll << 30)) return NQ_ERR_UNSUPPORTED;
+    if (!part_bit && (ldw < K || (ldw & 15))) return ldw < K ? NQ_ERR_INVALID_ARG : NQ_ERR_ALIGNMENT;
+    if (!aligned16(Wt) || !aligned16(X)) return NQ_ERR_ALIGNMENT;
+    const int64_t need = nq_conv_workspace_bytes(d);
+    if (need > 0 && (!workspace || workspace_bytes < need)) return NQ_ERR_WORKSPACE;
+    if (need > 0 && (reinterpret_cast<uintptr_t>(workspace) & 1023)) return NQ_ERR_ALIGNMENT;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    CUtensorMap tmA;
+
+    if (!implicit_ok(*d)) {
+        // explicit patch matrix, then the plain GEMM path
+        const int ld = (int)((K + 15) / 16 * 16);
+        const long long chunks = M * (ld / 16);
+        im2col_kernel<<<(unsigned)((chunks + 255) / 256), 256, 0, stream>>>(X, (int8_t*)workspace, *d, Ho, Wo, (int)K, ld, chunks);
+        if (cudaGetLastError() != cudaSuccess) return NQ_ERR_CUDA;
+        int st = encode_tensor_map_2d(&tmA, workspace, (uint64_t)K, (uint64_t)M, (uint64_t)ld, kBK, kBM, 128);
+        if (st != NQ_OK) return st;
+        return run_contraction(tmA, kModeGemm, nullptr, (int)((M + kBM - 1) / kBM), (int)((K + kBK - 1) / kBK), Wt, ldw,
+                               part_bit != 0, n_bits, h_bits, w_scale, act_scale, bias, M, N, K, acc_out, N, Y, N, y_dtype,
+                               stream);
+    }
+
+    const int8_t* x_nhwc = X;
+    if (d->x_nchw) {
+        const int HW = d->H * d->W;
+        dim3 grid((HW + 63) / 64, (d->Cin + 63) / 64, d->B);
+        nchw_to_nhwc_kernel<<<grid, 256, 0, stream>>>(X, (int8_t*)workspace, d->Cin, HW);
+        if (cudaGetLastError() != cudaSuccess) return NQ_ERR_CUDA;
+        x_nhwc = (const int8_t*)workspace;
+    }
+    ConvGeom g{};
+    g.B = d->B; g.Ho = Ho; g.Wo = Wo; g.S = d->S; g.taps = d->R * d->S; g.stride = d->stride; g.pad = d->pad;
+    choose_tile(d->B, Ho, Wo, g.tw_log2, g.th_log2);
+    const int tw = 1 << g.tw_log2, th = 1 << g.th_log2, tb = 128 >> (g.tw_log2 + g.th_log2);
+    g.tiles_w = (Wo + tw - 1) / tw;
+    g.tiles_h = (Ho + th - 1) / th;
+    const int tiles_b = (d->B + tb - 1) / tb;
+    const int m_tiles = g.tiles_w * g.tiles_h * tiles_b;
+    int mode, k_blocks, st;
+    if (d->Cin == 64) {
+        mode = kModeConv64;
+        g.cblocks = 1;
+        k_blocks = (g.taps + 1) / 2;
+        st = encode_tensor_map_nhwc(&tmA, x_nhwc, d->Cin, d->W, d->H, d->B, 64, tw, th, tb, d->stride, 64);
+    } else {
+        mode = kModeConv128;
+        g.cblocks = d->Cin / 128;
+        k_blocks = g.taps * g.cblocks;
+        st = encode_tensor_map_nhwc(&tmA, x_nhwc, d->Cin, d->W, d->H, d->B, 128, tw, th, tb, d->stride, 128);
+    }
+    if (st != NQ_OK) return st;
+    return run_contraction(tmA, mode, &g, m_tiles, k_blocks, Wt, ldw, part_bit != 0, n_bits, h_bits, w_scale, act_scale,
+                           bias, M, N, K, acc_out, N, Y, N, y_dtype, stream);
 }
 
 }  // extern "C"

@@ -9,64 +9,101 @@
 
 namespace nq {
 
-int encode_tensor_map_2d(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t pitch_bytes,
-                         uint32_t box_inner, uint32_t box_outer, bool swizzle128) {
-    typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                 const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+namespace {
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                             const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                             CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeFn encode_fn() {
     static EncodeFn fn = nullptr;
     if (!fn) {
         void* sym = nullptr;
         cudaDriverEntryPointQueryResult q;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess || !sym ||
             q != cudaDriverEntryPointSuccess)
-            return NQ_ERR_CUDA;
+            return nullptr;
         fn = reinterpret_cast<EncodeFn>(sym);
     }
+    return fn;
+}
+CUtensorMapSwizzle swizzle_of(int bytes) {
+    return bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE;
+}
+}  // namespace
+
+int encode_tensor_map_2d(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t pitch_bytes,
+                         uint32_t box_inner, uint32_t box_outer, int swizzle_bytes) {
+    EncodeFn fn = encode_fn();
+    if (!fn) return NQ_ERR_CUDA;
     cuuint64_t dims[2] = {inner, outer};
     cuuint64_t strides[1] = {pitch_bytes};
     cuuint32_t box[2] = {box_inner, box_outer};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
-                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_of(swizzle_bytes), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? NQ_OK : NQ_ERR_CUDA;
+}
+
+int encode_tensor_map_nhwc(CUtensorMap* map, const void* base, uint64_t C, uint64_t W, uint64_t H, uint64_t B,
+                           uint32_t box_c, uint32_t tw, uint32_t th, uint32_t tb, uint32_t stride, int swizzle_bytes) {
+    EncodeFn fn = encode_fn();
+    if (!fn) return NQ_ERR_CUDA;
+    cuuint64_t dims[4] = {C, W, H, B};
+    cuuint64_t strides[3] = {C, C * W, C * W * H};
+    // the box spans (t - 1) * stride + 1 input positions, of which every stride-th is taken: t elements
+    cuuint32_t box[4] = {box_c, (tw - 1) * stride + 1, (th - 1) * stride + 1, tb};
+    cuuint32_t estr[4] = {1, stride, stride, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_of(swizzle_bytes), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? NQ_OK : NQ_ERR_CUDA;
 }
 
 namespace {
 
-template <int BN, bool PART>
+template <int BN, bool PART, int MODE>
 int launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const ContractionArgs& a, cudaStream_t stream) {
     const int smem = contraction_smem_bytes(BN, PART, a.h_bits);
     static int configured[64] = {0};       // largest opt-in done so far, per device, for this instantiation
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return NQ_ERR_CUDA;
     if (smem > configured[dev]) {
-        if (cudaFuncSetAttribute(contraction_kernel<BN, PART>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
-            cudaSuccess)
+        if (cudaFuncSetAttribute(contraction_kernel<BN, PART, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 smem) != cudaSuccess)
             return NQ_ERR_CUDA;
         configured[dev] = smem;
     }
     const int tiles = a.m_tiles * a.n_tiles;
     const int grid = tiles < sm_count() ? tiles : sm_count();
-    contraction_kernel<BN, PART><<<grid, PART ? 320 : 192, smem, stream>>>(tmA, tmB, a);
+    contraction_kernel<BN, PART, MODE><<<grid, PART ? 320 : 192, smem, stream>>>(tmA, tmB, a);
     return cudaGetLastError() == cudaSuccess ? NQ_OK : NQ_ERR_CUDA;
+}
+
+template <int BN, bool PART>
+int launch_mode(int mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const ContractionArgs& a, cudaStream_t s) {
+    if (mode == kModeConv128) return launch<BN, PART, kModeConv128>(tmA, tmB, a, s);
+    if (mode == kModeConv64) return launch<BN, PART, kModeConv64>(tmA, tmB, a, s);
+    return launch<BN, PART, kModeGemm>(tmA, tmB, a, s);
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 }  // namespace
 
-// A is an int8 [M, K] matrix reached through tmA (built by the caller: plain 2-D for the GEMM).
-int run_contraction(const CUtensorMap& tmA, const void* Bmat, int64_t ldb, bool part, int n_bits, int h_bits,
+// The A operand is reached through tmA, built by the caller: a plain 2-D map of an [M, K] matrix
+// (kModeGemm, geom == nullptr) or a 4-D map of NHWC activations (convolution modes, geom given; then M
+// tiles are geom's pixel rectangles and k_blocks follows the filter taps).
+int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int m_tiles, int k_blocks,
+                    const void* Bmat, int64_t ldb, bool part, int n_bits, int h_bits,
                     const float* w_scale, float act_scale, const float* bias, int64_t M, int64_t N, int64_t K,
                     int32_t* acc_out, int64_t ld_acc, void* Y, int64_t ldy, int y_dtype, cudaStream_t stream) {
     const int bn = N > 128 ? 256 : (N > 64 ? 128 : 64);
     ContractionArgs a{};
+    if (geom) a.g = *geom;
     a.M = (int)M; a.N = (int)N; a.K = (int)K;
-    a.m_tiles = (int)((M + kBM - 1) / kBM);
+    a.m_tiles = m_tiles;
     a.n_tiles = (int)((N + bn - 1) / bn);
-    a.k_blocks = (int)((K + kBK - 1) / kBK);
+    a.k_blocks = k_blocks;
     a.w_scale = w_scale; a.bias = bias; a.act_scale = act_scale;
     a.acc_out = acc_out; a.ld_acc = ld_acc; a.y = Y; a.ldy = ldy; a.y_is_bf16 = (y_dtype == NQ_BF16);
     a.status = status_word();
@@ -78,22 +115,24 @@ int run_contraction(const CUtensorMap& tmA, const void* Bmat, int64_t ldb, bool 
         a.acc_shift = 8 - h_bits;
         a.unshift = 1.0f / (float)(1 << a.acc_shift);
         a.h_bits = h_bits;
-        const uint64_t row_bytes = (uint64_t)a.k_blocks * 16 * h_bits;
-        int st = encode_tensor_map_2d(&tmB, Bmat, row_bytes, (uint64_t)N, row_bytes, 16 * h_bits, bn, false);
+        const uint64_t row_bytes = (uint64_t)((K + 127) / 128) * 16 * h_bits;
+        int st = encode_tensor_map_2d(&tmB, Bmat, row_bytes, (uint64_t)N, row_bytes, 16 * h_bits, bn, 0);
         if (st != NQ_OK) return st;
     } else {
         a.pow2_l = 1.0f; a.unshift = 1.0f; a.acc_shift = 0; a.h_bits = 0;
-        int st = encode_tensor_map_2d(&tmB, Bmat, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, kBK, bn, true);
+        int st = (mode == kModeConv64)
+                     ? encode_tensor_map_2d(&tmB, Bmat, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, 64, bn, 64)
+                     : encode_tensor_map_2d(&tmB, Bmat, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, kBK, bn, 128);
         if (st != NQ_OK) return st;
     }
     if (part) {
-        if (bn == 256) return launch<256, true>(tmA, tmB, a, stream);
-        if (bn == 128) return launch<128, true>(tmA, tmB, a, stream);
-        return launch<64, true>(tmA, tmB, a, stream);
+        if (bn == 256) return launch_mode<256, true>(mode, tmA, tmB, a, stream);
+        if (bn == 128) return launch_mode<128, true>(mode, tmA, tmB, a, stream);
+        return launch_mode<64, true>(mode, tmA, tmB, a, stream);
     }
-    if (bn == 256) return launch<256, false>(tmA, tmB, a, stream);
-    if (bn == 128) return launch<128, false>(tmA, tmB, a, stream);
-    return launch<64, false>(tmA, tmB, a, stream);
+    if (bn == 256) return launch_mode<256, false>(mode, tmA, tmB, a, stream);
+    if (bn == 128) return launch_mode<128, false>(mode, tmA, tmB, a, stream);
+    return launch_mode<64, false>(mode, tmA, tmB, a, stream);
 }
 
 namespace {
@@ -115,10 +154,11 @@ int gemm_common(const int8_t* X, int64_t ldx, const void* Bmat, int64_t ldb, boo
     if ((acc_out && (reinterpret_cast<uintptr_t>(acc_out) & 3)) || (Y && (reinterpret_cast<uintptr_t>(Y) & 1)))
         return NQ_ERR_ALIGNMENT;
     CUtensorMap tmA;
-    int st = encode_tensor_map_2d(&tmA, X, (uint64_t)K, (uint64_t)M, (uint64_t)ldx, kBK, kBM, true);
+    int st = encode_tensor_map_2d(&tmA, X, (uint64_t)K, (uint64_t)M, (uint64_t)ldx, kBK, kBM, 128);
     if (st != NQ_OK) return st;
-    return run_contraction(tmA, Bmat, ldb, part, n_bits, h_bits, w_scale, act_scale, bias, M, N, K, acc_out, ld_acc, Y,
-                           ldy, y_dtype, (cudaStream_t)stream);
+    return run_contraction(tmA, kModeGemm, nullptr, (int)((M + kBM - 1) / kBM), (int)((K + kBK - 1) / kBK), Bmat, ldb,
+                           part, n_bits, h_bits, w_scale, act_scale, bias, M, N, K, acc_out, ld_acc, Y, ldy, y_dtype,
+                           (cudaStream_t)stream);
 }
 
 }  // namespace

@@ -13,3 +13,4 @@ int sm_count();
 unsigned int* status_word();
 
 }  // namespace nq
+

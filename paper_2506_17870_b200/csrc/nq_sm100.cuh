@@ -80,6 +80,14 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y)
         : "memory");
 }
+// 4-D tile load (channels, width, height, batch of an NHWC tensor); coordinates may lie outside the tensor,
+// where the copy writes zeros -- that is the convolution's zero padding.  No multicast.
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c, int w, int h, int n, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n)
+        : "memory");
+}
 // generic-proxy writes to shared memory -> visible to the async proxy (TMA, tcgen05.mma)
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -109,6 +117,10 @@ __device__ __forceinline__ void tc_fence_after_sync() {
 // descriptor version 1, layout type 2 (128-byte swizzle).
 __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
     return static_cast<uint64_t>((addr >> 4) & 0x3fffu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// The same for 64-byte rows in the 64-byte swizzle: 8-row groups are 512 B apart, layout type 4.
+__device__ __forceinline__ uint64_t smem_desc_sw64(uint32_t addr) {
+    return static_cast<uint64_t>((addr >> 4) & 0x3fffu) | (1ull << 16) | (32ull << 32) | (1ull << 46) | (4ull << 61);
 }
 // Instruction descriptor for kind::i8: D = S32, A = B = signed INT8, both K-major, M x N tile.
 __host__ __device__ constexpr uint32_t idesc_i8(int m, int n) {
@@ -154,7 +166,12 @@ __device__ __forceinline__ void named_barrier_sync(int id, int threads) {
 
 // Host: encode a 2-D tiled tensor map through the driver entry point (no link-time libcuda).
 // dims / box are {inner, outer}; pitch_bytes is the byte stride of the outer dimension.
+// swizzle_bytes is 0, 64 or 128.
 int encode_tensor_map_2d(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t pitch_bytes,
-                         uint32_t box_inner, uint32_t box_outer, bool swizzle128);
+                         uint32_t box_inner, uint32_t box_outer, int swizzle_bytes);
+// NHWC int8 activations as a 4-D tensor (C, W, H, B); the box covers box_c channels of tw x th x tb output
+// pixels taken every `stride` input pixels.
+int encode_tensor_map_nhwc(CUtensorMap* map, const void* base, uint64_t C, uint64_t W, uint64_t H, uint64_t B,
+                           uint32_t box_c, uint32_t tw, uint32_t th, uint32_t tb, uint32_t stride, int swizzle_bytes);
 
 }  // namespace nq
