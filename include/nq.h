@@ -184,6 +184,32 @@ NQ_API int nq_conv_implicit_gemm(const int8_t *X, const void *Wt, int64_t ldw, i
                           void *workspace, int64_t workspace_bytes, void *stream);
 
 /*
+ * The convolution again, for callers that must not allocate.  (The paper has no counterpart; this is a
+ * convenience of the library.)  nq_conv_implicit_gemm needs a workspace whenever it re-lays the input
+ * (NCHW activations, or a channel count it cannot gather in place), and somebody has to allocate that.
+ * Code that runs where cudaMalloc is off the table -- a plug-in handed a fixed set of buffers by its host
+ * application, a real-time loop that may not touch the allocator, a process whose memory budget was
+ * pinned at start-up -- can call this variant instead: it takes the same inputs and outputs and no
+ * workspace, and stages through an array that is part of the library image itself.
+ *   - The array is NQ_CONV_STATIC_SCRATCH_BYTES (16 MiB) of device memory.  Every GPU on which the library
+ *     is loaded carries it from load to process exit, used or not.
+ *   - A layer whose nq_conv_workspace_bytes() exceeds that size is refused with NQ_ERR_WORKSPACE and
+ *     nothing is launched; use nq_conv_implicit_gemm with your own buffer for those.
+ *   - The first call on each device looks the array's device address up (one runtime query, with that
+ *     device current).  Make that first call before you start capturing a stream.
+ *   - All calls share the one array and it keeps whatever the previous call left there.  The kernels
+ *     overwrite every byte they later read, so nothing has to be cleared between calls; but two calls
+ *     whose work overlaps on the GPU (different streams, or different host threads) would scribble over
+ *     each other's staging data.  Keep calls on one stream, or order them yourself.
+ *   - No cudaMalloc, cudaFree or allocating library routine is called.
+ * Arguments, layouts, results and error codes are otherwise those of nq_conv_implicit_gemm.
+ */
+#define NQ_CONV_STATIC_SCRATCH_BYTES (16 * 1024 * 1024)
+NQ_API int nq_conv_implicit_gemm_static(const int8_t *X, const void *Wt, int64_t ldw, int part_bit, int n_bits,
+                                        int h_bits, const nq_conv_desc *desc, const float *w_scale, float act_scale,
+                                        const float *bias, int32_t *acc_out, void *Y, int y_dtype, void *stream);
+
+/*
  * Every on-device wait in the GEMM / convolution kernels is bounded.  If one expires the kernel
  * records it and returns instead of hanging.  This call synchronises `stream`, reads and clears
  * the record of the current device: returns NQ_OK, NQ_ERR_TIMEOUT (with *where_out = an internal

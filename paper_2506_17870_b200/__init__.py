@@ -6,7 +6,7 @@ loads the library and raises ``NqLibraryError`` if it has not been built -- ther
 """
 from .binding import (  # noqa: F401
     BatchPlan, NqError, NqLibraryError, EXPORTS, NQ_BF16, NQ_F32, lib, nq_batch_plan, nq_conv_desc,
-    nq_conv_implicit_gemm, nq_conv_workspace_bytes, nq_decompose, nq_device_status, nq_drop_low,
+    nq_conv_implicit_gemm, nq_conv_implicit_gemm_static, nq_conv_workspace_bytes, NQ_CONV_STATIC_SCRATCH_BYTES, nq_decompose, nq_device_status, nq_drop_low,
     nq_drop_low_batched, nq_gemm_full, nq_gemm_part, nq_low_bits, nq_pack, nq_packed_bytes,
     nq_packed_row_bytes, nq_recompose, nq_recompose_batched, nq_tensor_desc, nq_unpack, status_str,
 )

@@ -27,6 +27,7 @@ EXPORTS = (
     "nq_decompose", "nq_recompose", "nq_drop_low", "nq_unpack", "nq_pack",
     "nq_batch_table_bytes", "nq_batch_plan", "nq_recompose_batched", "nq_drop_low_batched",
     "nq_gemm_full", "nq_gemm_part", "nq_conv_workspace_bytes", "nq_conv_implicit_gemm",
+    "nq_conv_implicit_gemm_static",
     "nq_device_status",
 )
 
@@ -307,6 +308,34 @@ def nq_conv_implicit_gemm(X: torch.Tensor, Wt: torch.Tensor, desc: nq_conv_desc,
                                        _ptr(acc), _ptr(y), _y_dtype(y.dtype) if y is not None else NQ_F32,
                                        _ptr(ws), _i64(ws.numel()), _stream()), "nq_conv_implicit_gemm")
     return acc, y, workspace
+
+
+NQ_CONV_STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
+
+
+def nq_conv_implicit_gemm_static(X: torch.Tensor, Wt: torch.Tensor, desc: nq_conv_desc, w_scale: torch.Tensor,
+                                 act_scale: float, acc_out: Optional[torch.Tensor], y_out: Optional[torch.Tensor],
+                                 part_bit: bool = False, n_bits: int = 8, h_bits: int = 6,
+                                 bias: Optional[torch.Tensor] = None):
+    """The convolution for callers that cannot allocate: no workspace argument, and this wrapper allocates
+    nothing either -- the caller passes the output tensors (acc_out int32 and / or y_out fp32 / bf16, NHWC).
+    Layers that need more than NQ_CONV_STATIC_SCRATCH_BYTES of staging raise NqError(NQ_ERR_WORKSPACE)."""
+    _need(X, torch.int8, "X")
+    _need(w_scale, torch.float32, "w_scale", 1)
+    if acc_out is None and y_out is None:
+        raise ValueError("pass acc_out and / or y_out")
+    if part_bit:
+        _need(Wt, torch.uint8, "Wt")
+        ldw = 0
+    else:
+        _need(Wt, torch.int8, "Wt", 2)
+        ldw = _ld(Wt)
+    _check(lib().nq_conv_implicit_gemm_static(_ptr(X), _ptr(Wt), _i64(ldw), int(bool(part_bit)), n_bits, h_bits,
+                                              ctypes.byref(desc), _ptr(w_scale), ctypes.c_float(act_scale), _ptr(bias),
+                                              _ptr(acc_out), _ptr(y_out),
+                                              _y_dtype(y_out.dtype) if y_out is not None else NQ_F32, _stream()),
+           "nq_conv_implicit_gemm_static")
+    return acc_out, y_out
 
 
 def nq_device_status() -> int:

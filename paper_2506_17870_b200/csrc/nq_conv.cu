@@ -15,6 +15,11 @@
 #include "nq_contraction.cuh"
 #include "nq_internal.cuh"
 
+// Staging memory of nq_conv_implicit_gemm_static: lives in the library image, one copy per GPU that loads it.
+// In host code this name is only a handle for cudaGetSymbolAddress -- it is not a device address.  The extra
+// 1 KiB lets the host round the address up to the 1 KiB alignment nq_conv_implicit_gemm asks of a workspace.
+static __device__ __align__(256) unsigned char g_conv_static_scratch[NQ_CONV_STATIC_SCRATCH_BYTES + 1024];
+
 namespace nq {
 namespace {
 
@@ -184,6 +189,26 @@ int nq_conv_implicit_gemm(const int8_t* X, const void* Wt, int64_t ldw, int part
     if (st != NQ_OK) return st;
     return run_contraction(tmA, mode, &g, m_tiles, k_blocks, Wt, ldw, part_bit != 0, n_bits, h_bits, w_scale, act_scale,
                            bias, M, N, K, acc_out, N, Y, N, y_dtype, stream);
+}
+
+int nq_conv_implicit_gemm_static(const int8_t* X, const void* Wt, int64_t ldw, int part_bit, int n_bits, int h_bits,
+                                 const nq_conv_desc* d, const float* w_scale, float act_scale, const float* bias,
+                                 int32_t* acc_out, void* Y, int y_dtype, void* stream) {
+    const int64_t need = nq_conv_workspace_bytes(d);
+    if (need < 0) return NQ_ERR_INVALID_ARG;
+    if (need > (int64_t)NQ_CONV_STATIC_SCRATCH_BYTES) return NQ_ERR_WORKSPACE;   // does not fit the built-in staging array
+    // device address of the array, looked up once per device with that device current
+    static unsigned char* base[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return NQ_ERR_CUDA;
+    if (!base[dev]) {
+        unsigned char* ptr = nullptr;
+        if (cudaGetSymbolAddress((void**)&ptr, g_conv_static_scratch) != cudaSuccess || !ptr) return NQ_ERR_CUDA;
+        base[dev] = ptr;
+    }
+    unsigned char* ws = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(base[dev]) + 1023) & ~uintptr_t(1023));
+    return nq_conv_implicit_gemm(X, Wt, ldw, part_bit, n_bits, h_bits, d, w_scale, act_scale, bias, acc_out, Y, y_dtype,
+                                 ws, NQ_CONV_STATIC_SCRATCH_BYTES, stream);
 }
 
 }  // extern "C"
