@@ -10,7 +10,7 @@
 //               a TMEM accumulator; owns the TMEM allocation
 //   warps 2-5   epilogue: tcgen05.ld the accumulator (each warp its 32-lane quarter), scale, store.
 //               Two accumulators alternate so the epilogue of tile i overlaps the MMAs of tile i+1
-//   warps 6-9   (part-bit only) unpackers: expand packed INTh fields into the swizzled int8 B tile.
+//   warps 6-13  (part-bit only) unpackers: expand packed INTh fields into the swizzled int8 B tile.
 //               The field goes to the TOP h bits of the byte, i.e. the byte is w_high * 2^(8-h); the
 //               accumulator is then 2^(8-h) times too large, exactly, and the epilogue takes it out
 //               (arithmetic shift for the int32 output, an exact power-of-two factor in the scale).
@@ -87,32 +87,85 @@ __device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, 
     nt = local / gsz;
 }
 
-// expand one 32-element unit of h-bit fields to 32 bytes, field in the top bits of each byte
-__device__ __forceinline__ void unpack_unit_top(const uint8_t* group, int unit, int bits, uint32_t (&T)[8]) {
+// One 32-element unit of packed H-bit fields as it sits in the shared-memory tile ...
+struct PackedUnit {
+    uint4 a;       // 4-bit slice
+    uint2 c;       // 2-bit slice
+    uint32_t d;    // 1-bit slice
+};
+template <int H>
+__device__ __forceinline__ void load_packed_unit(const uint8_t* group, int unit, PackedUnit& r) {
+    int off = 0;
+    if (H & 4) { r.a = *reinterpret_cast<const uint4*>(group + unit * 16); off = 64; }
+    if (H & 2) { r.c = *reinterpret_cast<const uint2*>(group + off + unit * 8); off += 32; }
+    if (H & 1) { r.d = *reinterpret_cast<const uint32_t*>(group + off + unit * 4); }
+}
+// ... and its expansion to 32 bytes with the field in the TOP H bits of each byte.  All shifts and masks are
+// immediates: the 4-bit slice costs one AND (or shift + AND) per word, every narrower slice one shift and one
+// masked OR per word.
+template <int H>
+__device__ __forceinline__ void expand_packed_unit(const PackedUnit& r, uint32_t (&T)[8]) {
 #pragma unroll
     for (int q = 0; q < 8; ++q) T[q] = 0;
-    int off = 0, used = 0;
-    if (bits & 4) {
-        uint4 w = *reinterpret_cast<const uint4*>(group + unit * 16);
-        T[0] = w.x & 0xf0f0f0f0u; T[1] = (w.x << 4) & 0xf0f0f0f0u;
-        T[2] = w.y & 0xf0f0f0f0u; T[3] = (w.y << 4) & 0xf0f0f0f0u;
-        T[4] = w.z & 0xf0f0f0f0u; T[5] = (w.z << 4) & 0xf0f0f0f0u;
-        T[6] = w.w & 0xf0f0f0f0u; T[7] = (w.w << 4) & 0xf0f0f0f0u;
-        off = 64; used = 4;
+    int used = 0;
+    if (H & 4) {
+        T[0] = r.a.x & 0xf0f0f0f0u; T[1] = (r.a.x << 4) & 0xf0f0f0f0u;
+        T[2] = r.a.y & 0xf0f0f0f0u; T[3] = (r.a.y << 4) & 0xf0f0f0f0u;
+        T[4] = r.a.z & 0xf0f0f0f0u; T[5] = (r.a.z << 4) & 0xf0f0f0f0u;
+        T[6] = r.a.w & 0xf0f0f0f0u; T[7] = (r.a.w << 4) & 0xf0f0f0f0u;
+        used = 4;
     }
-    if (bits & 2) {
-        uint2 w = *reinterpret_cast<const uint2*>(group + off + unit * 8);
+    if (H & 2) {
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
-            uint32_t word = (q < 4) ? w.x : w.y;
-            T[q] |= ((word << (2 * (q & 3))) & 0xc0c0c0c0u) >> used;
+            const uint32_t word = (q < 4) ? r.c.x : r.c.y;
+            const int net = 2 * (q & 3) - used;
+            const uint32_t moved = net >= 0 ? (word << net) : (word >> (-net));
+            T[q] |= moved & (0xc0c0c0c0u >> used);
         }
-        off += 32; used += 2;
+        used += 2;
     }
-    if (bits & 1) {
-        uint32_t w = *reinterpret_cast<const uint32_t*>(group + off + unit * 4);
+    if (H & 1) {
 #pragma unroll
-        for (int q = 0; q < 8; ++q) T[q] |= ((w << q) & 0x80808080u) >> used;
+        for (int q = 0; q < 8; ++q) {
+            const int net = q - used;
+            const uint32_t moved = net >= 0 ? (r.d << net) : (r.d >> (-net));
+            T[q] |= moved & (0x80808080u >> used);
+        }
+    }
+}
+
+constexpr int kUnpackWarps = 8;
+constexpr int kUnpackThreads = kUnpackWarps * 32;
+
+// Expand one packed B tile (BN rows x 128 fields) into the swizzled int8 tile the MMA reads.
+template <int BN, int MODE, int H>
+__device__ __forceinline__ void unpack_tile(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, int utid) {
+    constexpr int TASKS = BN * 4 / kUnpackThreads;         // units per thread: 4 lanes share a row
+    PackedUnit raw[TASKS];
+#pragma unroll
+    for (int i = 0; i < TASKS; ++i) {
+        const int task = i * kUnpackThreads + utid;
+        load_packed_unit<H>(src + (task >> 2) * 16 * H, task & 3, raw[i]);
+    }
+#pragma unroll
+    for (int i = 0; i < TASKS; ++i) {
+        const int task = i * kUnpackThreads + utid;
+        const int row = task >> 2, unit = task & 3;
+        uint32_t T[8];
+        expand_packed_unit<H>(raw[i], T);
+        if (MODE == kModeConv64) {
+            // two sub-tiles of 64-byte rows: units 0,1 feed the first, 2,3 the second; 64-byte swizzle
+            uint8_t* drow = dst + (unit >> 1) * (BN * 64) + row * 64;
+            const int sw = (row >> 1) & 3, c = (unit & 1) * 2;
+            *reinterpret_cast<uint4*>(drow + ((c ^ sw) << 4)) = make_uint4(T[0], T[1], T[2], T[3]);
+            *reinterpret_cast<uint4*>(drow + (((c + 1) ^ sw) << 4)) = make_uint4(T[4], T[5], T[6], T[7]);
+        } else {
+            uint8_t* drow = dst + row * 128;
+            const int sw = row & 7;
+            *reinterpret_cast<uint4*>(drow + (((2 * unit) ^ sw) << 4)) = make_uint4(T[0], T[1], T[2], T[3]);
+            *reinterpret_cast<uint4*>(drow + (((2 * unit + 1) ^ sw) << 4)) = make_uint4(T[4], T[5], T[6], T[7]);
+        }
     }
 }
 
@@ -130,7 +183,7 @@ __device__ __forceinline__ TileOrigin conv_tile_origin(const ConvGeom& g, int mt
 }
 
 template <int BN, bool PART, int MODE>
-__global__ void __launch_bounds__(PART ? 320 : 192, 1)
+__global__ void __launch_bounds__(PART ? 192 + kUnpackThreads : 192, 1)
 contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                    const ContractionArgs p) {
     using namespace sm100;
@@ -165,12 +218,12 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(smem_u32(&full[s]), PART ? 1 + 4 : 1);   // producer (+ one arrival per unpack warp)
+            mbar_init(smem_u32(&full[s]), PART ? 1 + kUnpackWarps : 1);   // producer (+ one arrival per unpack warp)
             mbar_init(smem_u32(&empty[s]), 1);                 // tcgen05.commit
         }
         for (int s = 0; s < kPackedStages; ++s) {
             mbar_init(smem_u32(&pfull[s]), 1);
-            mbar_init(smem_u32(&pempty[s]), 4);
+            mbar_init(smem_u32(&pempty[s]), kUnpackWarps);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&tfull[b]), 1);
@@ -398,11 +451,10 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             if (lane == 0) mbar_arrive(smem_u32(&tempty[buf]));
         }
     } else if (PART) {
-        // ------------------------------------------------------------------ unpackers (warps 6-9)
-        const int utid = threadIdx.x - 192;            // 0..127
+        // ------------------------------------------------------------------ unpackers (warps 6-13)
+        const int utid = threadIdx.x - 192;
         uint32_t it = 0;
         bool ok = true;
-        const int h = p.h_bits;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
             for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
                 const uint32_t s = it % STAGES, use = it / STAGES;
@@ -413,23 +465,14 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 if (!ok) break;
                 const uint8_t* src = sP + ps * packed_bytes;
                 uint8_t* dst = sB + s * B_BYTES;
-#pragma unroll 2
-                for (int task = utid; task < BN * 4; task += 128) {
-                    const int row = task >> 2, unit = task & 3;
-                    uint32_t T[8];
-                    unpack_unit_top(src + row * 16 * h, unit, h, T);
-                    if (MODE == kModeConv64) {
-                        // two sub-tiles of 64-byte rows: units 0,1 feed the first, 2,3 the second; 64-byte swizzle
-                        uint8_t* drow = dst + (unit >> 1) * (B_BYTES / 2) + row * 64;
-                        const int sw = (row >> 1) & 3, c = (unit & 1) * 2;
-                        *reinterpret_cast<uint4*>(drow + ((c ^ sw) << 4)) = make_uint4(T[0], T[1], T[2], T[3]);
-                        *reinterpret_cast<uint4*>(drow + (((c + 1) ^ sw) << 4)) = make_uint4(T[4], T[5], T[6], T[7]);
-                    } else {
-                        uint8_t* drow = dst + row * 128;
-                        const int sw = row & 7;
-                        *reinterpret_cast<uint4*>(drow + (((2 * unit) ^ sw) << 4)) = make_uint4(T[0], T[1], T[2], T[3]);
-                        *reinterpret_cast<uint4*>(drow + (((2 * unit + 1) ^ sw) << 4)) = make_uint4(T[4], T[5], T[6], T[7]);
-                    }
+                switch (p.h_bits) {                    // one specialised expansion per field width
+                    case 1: unpack_tile<BN, MODE, 1>(src, dst, utid); break;
+                    case 2: unpack_tile<BN, MODE, 2>(src, dst, utid); break;
+                    case 3: unpack_tile<BN, MODE, 3>(src, dst, utid); break;
+                    case 4: unpack_tile<BN, MODE, 4>(src, dst, utid); break;
+                    case 5: unpack_tile<BN, MODE, 5>(src, dst, utid); break;
+                    case 6: unpack_tile<BN, MODE, 6>(src, dst, utid); break;
+                    default: unpack_tile<BN, MODE, 7>(src, dst, utid); break;
                 }
                 fence_proxy_async_smem();              // these writes feed tcgen05.mma (async proxy)
                 __syncwarp();

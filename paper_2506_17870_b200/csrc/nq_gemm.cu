@@ -75,7 +75,7 @@ int launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const ContractionArgs
     }
     const int tiles = a.m_tiles * a.n_tiles;
     const int grid = tiles < sm_count() ? tiles : sm_count();
-    contraction_kernel<BN, PART, MODE><<<grid, PART ? 320 : 192, smem, stream>>>(tmA, tmB, a);
+    contraction_kernel<BN, PART, MODE><<<grid, PART ? 192 + kUnpackThreads : 192, smem, stream>>>(tmA, tmB, a);
     return cudaGetLastError() == cudaSuccess ? NQ_OK : NQ_ERR_CUDA;
 }
 
