@@ -15,7 +15,8 @@
 //               accumulator is then 2^(8-h) times too large, exactly, and the epilogue takes it out
 //               (arithmetic shift for the int32 output, an exact power-of-two factor in the scale).
 // Every mbarrier wait is bounded (see mbar_wait); when one gives up every role leaves its loop,
-// the block joins, frees its TMEM and returns, and the host can read the record.
+// the block joins, frees its TMEM and returns, and the host can read the record.  Every TMA load
+// has a single destination CTA.
 #pragma once
 #include <cuda_bf16.h>
 
@@ -27,7 +28,7 @@ constexpr int kBM = 128;           // tile rows (M) = TMEM lanes
 constexpr int kBK = 128;           // K bytes per stage = one 128-byte swizzle row
 constexpr int kStagesFull = 4;
 constexpr int kStagesPart = 3;
-constexpr int kPackedStages = 2;
+constexpr int kMaxPackedStages = 8;     // ring of packed (still INTh) B tiles; the depth in use is chosen by the host
 constexpr int kGroupM = 16;        // tile rasterisation: 16 M-tiles share a band of N-tiles
 
 // How the A operand is gathered.
@@ -56,6 +57,7 @@ struct ContractionArgs {
     float unshift;       // 2^-(8-h) in part-bit mode, 1 otherwise (exact)
     int acc_shift;       // 8-h in part-bit mode, 0 otherwise
     int h_bits;          // part-bit: width of the packed field
+    int packed_stages;   // part-bit: depth of the packed-tile ring (1..kMaxPackedStages)
     int32_t* acc_out;
     long long ld_acc;
     void* y;
@@ -68,12 +70,14 @@ __host__ __device__ constexpr int a_stage_bytes() { return kBM * kBK; }
 __host__ __device__ constexpr int b_stage_bytes(int bn) { return bn * kBK; }
 
 // dynamic shared memory: [A stages][B stages][packed stages][scale + bias per epilogue warp][barriers]
-__host__ __device__ inline int contraction_smem_bytes(int bn, bool part, int h_bits) {
+constexpr int kSmemLimit = 227 * 1024;   // dynamic shared memory a block may opt in to
+
+__host__ __device__ inline int contraction_smem_bytes(int bn, bool part, int h_bits, int packed_stages) {
     int stages = part ? kStagesPart : kStagesFull;
     int bytes = stages * (a_stage_bytes() + b_stage_bytes(bn));
-    if (part) bytes += kPackedStages * bn * 16 * h_bits;
+    if (part) bytes += packed_stages * bn * 16 * h_bits;
     bytes += 4 * 2 * bn * (int)sizeof(float);   // scale and bias, one private copy per epilogue warp
-    bytes += 256;                       // barriers, TMEM base, abort flag
+    bytes += 512;                       // barriers, TMEM base, abort flag
     return bytes + 1024;                // slack to align the base to 1024 B
 }
 
@@ -138,33 +142,39 @@ __device__ __forceinline__ void expand_packed_unit(const PackedUnit& r, uint32_t
 constexpr int kUnpackWarps = 8;
 constexpr int kUnpackThreads = kUnpackWarps * 32;
 
-// Expand one packed B tile (BN rows x 128 fields) into the swizzled int8 tile the MMA reads.
-template <int BN, int MODE, int H>
-__device__ __forceinline__ void unpack_tile(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, int utid) {
-    constexpr int TASKS = BN * 4 / kUnpackThreads;         // units per thread: 4 lanes share a row
-    PackedUnit raw[TASKS];
+// Expand one packed B tile (ROWS rows x 128 fields) into the swizzled int8 tile the MMA reads, with THREADS
+// threads (tid = 0 .. THREADS-1); four consecutive threads share a row.
+template <int ROWS, int MODE, int H, int THREADS>
+__device__ __forceinline__ void unpack_tile(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, int tid) {
+    constexpr int TASKS = ROWS * 4 / THREADS;              // units per thread
+    constexpr int CHUNK = TASKS < 4 ? TASKS : 4;           // units whose loads are issued together
+    static_assert(TASKS >= 1 && TASKS % CHUNK == 0, "tile does not divide over the threads");
 #pragma unroll
-    for (int i = 0; i < TASKS; ++i) {
-        const int task = i * kUnpackThreads + utid;
-        load_packed_unit<H>(src + (task >> 2) * 16 * H, task & 3, raw[i]);
-    }
+    for (int base = 0; base < TASKS; base += CHUNK) {
+        PackedUnit raw[CHUNK];
 #pragma unroll
-    for (int i = 0; i < TASKS; ++i) {
-        const int task = i * kUnpackThreads + utid;
-        const int row = task >> 2, unit = task & 3;
-        uint32_t T[8];
-        expand_packed_unit<H>(raw[i], T);
-        if (MODE == kModeConv64) {
-            // two sub-tiles of 64-byte rows: units 0,1 feed the first, 2,3 the second; 64-byte swizzle
-            uint8_t* drow = dst + (unit >> 1) * (BN * 64) + row * 64;
-            const int sw = (row >> 1) & 3, c = (unit & 1) * 2;
-            *reinterpret_cast<uint4*>(drow + ((c ^ sw) << 4)) = make_uint4(T[0], T[1], T[2], T[3]);
-            *reinterpret_cast<uint4*>(drow + (((c + 1) ^ sw) << 4)) = make_uint4(T[4], T[5], T[6], T[7]);
-        } else {
-            uint8_t* drow = dst + row * 128;
-            const int sw = row & 7;
-            *reinterpret_cast<uint4*>(drow + (((2 * unit) ^ sw) << 4)) = make_uint4(T[0], T[1], T[2], T[3]);
-            *reinterpret_cast<uint4*>(drow + (((2 * unit + 1) ^ sw) << 4)) = make_uint4(T[4], T[5], T[6], T[7]);
+        for (int i = 0; i < CHUNK; ++i) {
+            const int task = (base + i) * THREADS + tid;
+            load_packed_unit<H>(src + (task >> 2) * 16 * H, task & 3, raw[i]);
+        }
+#pragma unroll
+        for (int i = 0; i < CHUNK; ++i) {
+            const int task = (base + i) * THREADS + tid;
+            const int row = task >> 2, unit = task & 3;
+            uint32_t T[8];
+            expand_packed_unit<H>(raw[i], T);
+            if (MODE == kModeConv64) {
+                // two sub-tiles of 64-byte rows: units 0,1 feed the first, 2,3 the second; 64-byte swizzle
+                uint8_t* drow = dst + (unit >> 1) * (ROWS * 64) + row * 64;
+                const int sw = (row >> 1) & 3, c = (unit & 1) * 2;
+                *reinterpret_cast<uint4*>(drow + ((c ^ sw) << 4)) = make_uint4(T[0], T[1], T[2], T[3]);
+                *reinterpret_cast<uint4*>(drow + (((c + 1) ^ sw) << 4)) = make_uint4(T[4], T[5], T[6], T[7]);
+            } else {
+                uint8_t* drow = dst + row * 128;
+                const int sw = row & 7;
+                *reinterpret_cast<uint4*>(drow + (((2 * unit) ^ sw) << 4)) = make_uint4(T[0], T[1], T[2], T[3]);
+                *reinterpret_cast<uint4*>(drow + (((2 * unit + 1) ^ sw) << 4)) = make_uint4(T[4], T[5], T[6], T[7]);
+            }
         }
     }
 }
@@ -180,6 +190,69 @@ __device__ __forceinline__ TileOrigin conv_tile_origin(const ConvGeom& g, int mt
     o.p0 = (rest % g.tiles_h) << g.th_log2;
     o.b0 = (rest / g.tiles_h) << (7 - g.tw_log2 - g.th_log2);
     return o;
+}
+
+// Epilogue of one thread for 32 consecutive columns of its output row: optional int32 copy (with the
+// part-bit shift), dequantisation in the stated rounding order, fp32 or bf16 store; vector stores when
+// the chunk is whole and the pointers and pitches allow.
+__device__ __forceinline__ void store_chunk(const ContractionArgs& p, long long row, int col0, const uint32_t (&r)[32],
+                                            const float* sc, const float* bs, bool vec_acc, bool vec_f32, bool vec_bf16) {
+    const bool full_chunk = col0 + 32 <= p.N;
+    if (p.acc_out) {
+        int32_t* dst = p.acc_out + row * p.ld_acc + col0;
+        if (full_chunk && vec_acc) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<int4*>(dst + j) =
+                    make_int4((int)r[j] >> p.acc_shift, (int)r[j + 1] >> p.acc_shift,
+                              (int)r[j + 2] >> p.acc_shift, (int)r[j + 3] >> p.acc_shift);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (col0 + j < p.N) dst[j] = (int)r[j] >> p.acc_shift;
+        }
+    }
+    if (p.y) {
+        float v[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            float t = __fmul_rn(__int2float_rn((int)r[j]), sc[j]);
+            v[j] = p.bias ? __fadd_rn(t, bs[j]) : t;
+        }
+        if (!p.y_is_bf16) {
+            float* dst = reinterpret_cast<float*>(p.y) + row * p.ldy + col0;
+            if (full_chunk && vec_f32) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 4)
+                    *reinterpret_cast<float4*>(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                    if (col0 + j < p.N) dst[j] = v[j];
+            }
+        } else {
+            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.y) + row * p.ldy + col0;
+            if (full_chunk && vec_bf16) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) {
+                    __nv_bfloat162 a = __floats2bfloat162_rn(v[j], v[j + 1]);
+                    __nv_bfloat162 b = __floats2bfloat162_rn(v[j + 2], v[j + 3]);
+                    __nv_bfloat162 c2 = __floats2bfloat162_rn(v[j + 4], v[j + 5]);
+                    __nv_bfloat162 d = __floats2bfloat162_rn(v[j + 6], v[j + 7]);
+                    uint4 o;
+                    o.x = *reinterpret_cast<uint32_t*>(&a);
+                    o.y = *reinterpret_cast<uint32_t*>(&b);
+                    o.z = *reinterpret_cast<uint32_t*>(&c2);
+                    o.w = *reinterpret_cast<uint32_t*>(&d);
+                    *reinterpret_cast<uint4*>(dst + j) = o;
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                    if (col0 + j < p.N) dst[j] = __float2bfloat16_rn(v[j]);
+            }
+        }
+    }
 }
 
 template <int BN, bool PART, int MODE>
@@ -199,15 +272,15 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     uint8_t* sB = sA + STAGES * A_BYTES;
     const int packed_bytes = PART ? BN * 16 * p.h_bits : 0;
     uint8_t* sP = sB + STAGES * B_BYTES;
-    float* sScale = reinterpret_cast<float*>(sP + (PART ? kPackedStages * packed_bytes : 0));   // [4 warps][BN]
+    float* sScale = reinterpret_cast<float*>(sP + (PART ? p.packed_stages * packed_bytes : 0));   // [4 warps][BN]
     float* sBias = sScale + 4 * BN;                                                             // [4 warps][BN]
     uint64_t* bars = reinterpret_cast<uint64_t*>(sBias + 4 * BN);
     // barrier map: full[STAGES], empty[STAGES], pfull[2], pempty[2], tfull[2], tempty[2]
     uint64_t* full = bars;
     uint64_t* empty = full + STAGES;
     uint64_t* pfull = empty + STAGES;
-    uint64_t* pempty = pfull + kPackedStages;
-    uint64_t* tfull = pempty + kPackedStages;
+    uint64_t* pempty = pfull + kMaxPackedStages;
+    uint64_t* tfull = pempty + kMaxPackedStages;
     uint64_t* tempty = tfull + 2;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -221,7 +294,7 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             mbar_init(smem_u32(&full[s]), PART ? 1 + kUnpackWarps : 1);   // producer (+ one arrival per unpack warp)
             mbar_init(smem_u32(&empty[s]), 1);                 // tcgen05.commit
         }
-        for (int s = 0; s < kPackedStages; ++s) {
+        for (int s = 0; s < kMaxPackedStages; ++s) {
             mbar_init(smem_u32(&pfull[s]), 1);
             mbar_init(smem_u32(&pempty[s]), kUnpackWarps);
         }
@@ -246,7 +319,7 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            uint32_t it = 0, pit = 0;
+            uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
                 int mt, nt;
@@ -274,12 +347,7 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                         }
                     }
                     if (PART) {
-                        const uint32_t ps = pit % kPackedStages, puse = pit / kPackedStages;
-                        if (!(ok = mbar_wait(smem_u32(&pempty[ps]), (puse & 1) ^ 1, abort_flag, p.status, 0x11u))) break;
-                        const uint32_t pb = smem_u32(&pfull[ps]);
-                        mbar_arrive_expect_tx(pb, packed_bytes);
-                        tma_load_2d(smem_u32(sP + ps * packed_bytes), &tmB, kb * 16 * p.h_bits, nt * BN, pb);
-                        ++pit;
+                        // the packed tiles have a ring and a producer lane of their own (below)
                     } else if (MODE == kModeConv64) {
                         for (int sub = 0; sub < n_sub; ++sub)
                             tma_load_2d(smem_u32(sB + s * B_BYTES + sub * (B_BYTES / 2)), &tmB, kb * kBK + sub * 64, nt * BN, fb);
@@ -290,6 +358,26 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             }
             if (!ok) {
                 // gave up: let the copies already in flight land before the block releases its shared memory
+                const long long t0 = clock64();
+                while (clock64() - t0 < (1ll << 22)) { }
+            }
+        } else if (PART && lane == 1) {
+            // ---- packed-tile producer: runs ahead of the A loads by up to the depth of its own ring, which
+            //      is what hides the latency of fetching the weights
+            uint32_t pit = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+                int mt, nt;
+                tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++pit) {
+                    const uint32_t ps = pit % p.packed_stages, puse = pit / p.packed_stages;
+                    if (!(ok = mbar_wait(smem_u32(&pempty[ps]), (puse & 1) ^ 1, abort_flag, p.status, 0x11u))) break;
+                    const uint32_t pb = smem_u32(&pfull[ps]);
+                    mbar_arrive_expect_tx(pb, packed_bytes);
+                    tma_load_2d(smem_u32(sP + ps * packed_bytes), &tmB, kb * 16 * p.h_bits, nt * BN, pb);
+                }
+            }
+            if (!ok) {
                 const long long t0 = clock64();
                 while (clock64() - t0 < (1ll << 22)) { }
             }
@@ -387,64 +475,7 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 tmem_ld_wait();
                 const int col0 = n0 + c * 32;
                 if (!row_ok || col0 >= p.N) continue;
-                const float* sc = sc_w + c * 32;
-                const float* bs = bs_w + c * 32;
-                const bool full_chunk = col0 + 32 <= p.N;
-                if (p.acc_out) {
-                    int32_t* dst = p.acc_out + row * p.ld_acc + col0;
-                    if (full_chunk && vec_acc) {
-#pragma unroll
-                        for (int j = 0; j < 32; j += 4)
-                            *reinterpret_cast<int4*>(dst + j) =
-                                make_int4((int)r[j] >> p.acc_shift, (int)r[j + 1] >> p.acc_shift,
-                                          (int)r[j + 2] >> p.acc_shift, (int)r[j + 3] >> p.acc_shift);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (col0 + j < p.N) dst[j] = (int)r[j] >> p.acc_shift;
-                    }
-                }
-                if (p.y) {
-                    float v[32];
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        float t = __fmul_rn(__int2float_rn((int)r[j]), sc[j]);
-                        v[j] = p.bias ? __fadd_rn(t, bs[j]) : t;
-                    }
-                    if (!p.y_is_bf16) {
-                        float* dst = reinterpret_cast<float*>(p.y) + row * p.ldy + col0;
-                        if (full_chunk && vec_f32) {
-#pragma unroll
-                            for (int j = 0; j < 32; j += 4)
-                                *reinterpret_cast<float4*>(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (col0 + j < p.N) dst[j] = v[j];
-                        }
-                    } else {
-                        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.y) + row * p.ldy + col0;
-                        if (full_chunk && vec_bf16) {
-#pragma unroll
-                            for (int j = 0; j < 32; j += 8) {
-                                __nv_bfloat162 a = __floats2bfloat162_rn(v[j], v[j + 1]);
-                                __nv_bfloat162 b = __floats2bfloat162_rn(v[j + 2], v[j + 3]);
-                                __nv_bfloat162 c2 = __floats2bfloat162_rn(v[j + 4], v[j + 5]);
-                                __nv_bfloat162 d = __floats2bfloat162_rn(v[j + 6], v[j + 7]);
-                                uint4 o;
-                                o.x = *reinterpret_cast<uint32_t*>(&a);
-                                o.y = *reinterpret_cast<uint32_t*>(&b);
-                                o.z = *reinterpret_cast<uint32_t*>(&c2);
-                                o.w = *reinterpret_cast<uint32_t*>(&d);
-                                *reinterpret_cast<uint4*>(dst + j) = o;
-                            }
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (col0 + j < p.N) dst[j] = __float2bfloat16_rn(v[j]);
-                        }
-                    }
-                }
+                store_chunk(p, row, col0, r, sc_w + c * 32, bs_w + c * 32, vec_acc, vec_f32, vec_bf16);
             }
             tc_fence_before_sync();
             __syncwarp();
@@ -458,7 +489,7 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
             for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
                 const uint32_t s = it % STAGES, use = it / STAGES;
-                const uint32_t ps = it % kPackedStages, puse = it / kPackedStages;
+                const uint32_t ps = it % p.packed_stages, puse = it / p.packed_stages;
                 ok = mbar_wait(smem_u32(&pfull[ps]), puse & 1, abort_flag, p.status, 0x40u) &&
                      mbar_wait(smem_u32(&empty[s]), (use & 1) ^ 1, abort_flag, p.status, 0x41u);
                 ok = __all_sync(0xffffffffu, ok);
@@ -466,13 +497,13 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 const uint8_t* src = sP + ps * packed_bytes;
                 uint8_t* dst = sB + s * B_BYTES;
                 switch (p.h_bits) {                    // one specialised expansion per field width
-                    case 1: unpack_tile<BN, MODE, 1>(src, dst, utid); break;
-                    case 2: unpack_tile<BN, MODE, 2>(src, dst, utid); break;
-                    case 3: unpack_tile<BN, MODE, 3>(src, dst, utid); break;
-                    case 4: unpack_tile<BN, MODE, 4>(src, dst, utid); break;
-                    case 5: unpack_tile<BN, MODE, 5>(src, dst, utid); break;
-                    case 6: unpack_tile<BN, MODE, 6>(src, dst, utid); break;
-                    default: unpack_tile<BN, MODE, 7>(src, dst, utid); break;
+                    case 1: unpack_tile<BN, MODE, 1, kUnpackThreads>(src, dst, utid); break;
+                    case 2: unpack_tile<BN, MODE, 2, kUnpackThreads>(src, dst, utid); break;
+                    case 3: unpack_tile<BN, MODE, 3, kUnpackThreads>(src, dst, utid); break;
+                    case 4: unpack_tile<BN, MODE, 4, kUnpackThreads>(src, dst, utid); break;
+                    case 5: unpack_tile<BN, MODE, 5, kUnpackThreads>(src, dst, utid); break;
+                    case 6: unpack_tile<BN, MODE, 6, kUnpackThreads>(src, dst, utid); break;
+                    default: unpack_tile<BN, MODE, 7, kUnpackThreads>(src, dst, utid); break;
                 }
                 fence_proxy_async_smem();              // these writes feed tcgen05.mma (async proxy)
                 __syncwarp();

@@ -1,0 +1,322 @@
+// The INT8 contraction on CTA pairs (tcgen05 cta_group::2): 256 x 256 output tiles.
+//
+// Why pairs: with one CTA per 128 x 256 tile every K = 128 stage moves 48 KB into shared memory and the
+// tensor core reads 48 KB back out in 512 cycles -- the shared-memory port, not the tensor core, sets the
+// pace (measured: ~66 % tensor-pipe activity).  In a pair each CTA stages its own 128 rows of A and only
+// HALF of the B tile (128 of 256 rows); the tensor cores of both SMs read the two halves of B from both
+// shared memories.  Per SM that is 32 KB in and 32 KB out per stage, and in part-bit mode each SM unpacks
+// half as many weights.
+//
+// Roles per CTA are those of the single-CTA kernel (nq_contraction.cuh): warp 0 TMA producer, warp 1 MMA
+// issuer (only in the even, "leader" CTA; it also owns the TMEM allocation in both), warps 2-5 epilogue,
+// warps 6-13 unpackers (part-bit).  Barrier protocol, all barriers at the same offsets in both CTAs:
+//   full[s]    lives in the leader: 1 arrival by the leader's producer, which announces the bytes of BOTH
+//              CTAs' loads; the partner's loads complete on it through its cluster address; in part-bit
+//              mode the unpack warps of both CTAs arrive on it too
+//   empty[s]   one per CTA, arrived on in both CTAs at once by the leader's tcgen05.commit
+//   tfull[b]   likewise (accumulator b complete)
+//   tempty[b]  lives in the leader: the epilogue warps of both CTAs arrive (8 arrivals)
+//   pfull / pempty  packed-tile ring, private to each CTA
+// Every wait is bounded; every TMA load has a single destination CTA.
+#pragma once
+#include "nq_contraction.cuh"
+
+namespace nq {
+
+constexpr int kPairBN = 256;              // tile columns
+constexpr int kPairStagesFull = 6;
+constexpr int kPairStagesPart = 4;
+// The unpack warps work in groups: group g expands the stages whose counter is g modulo the group count, so a
+// group has that many stage times for one tile and the fixed per-stage costs (waits, proxy fence, the arrival
+// on the leader's barrier across the cluster) of different stages overlap.  Ring depths are multiples of the
+// group count, so that a ring slot is always served by the same group, in order: a parity wait is only valid
+// for a waiter that is at most one phase behind.
+constexpr int kUnpackGroups = 4;
+constexpr int kUnpackGroupWarps = kUnpackWarps / kUnpackGroups;
+constexpr int kUnpackGroupThreads = kUnpackGroupWarps * 32;
+static_assert(kPairStagesPart % kUnpackGroups == 0, "a stage slot must belong to one unpack group");
+
+__host__ __device__ inline int pair_smem_bytes(bool part, int h_bits, int packed_stages) {
+    const int stages = part ? kPairStagesPart : kPairStagesFull;
+    int bytes = stages * (a_stage_bytes() + b_stage_bytes(kPairBN / 2));
+    if (part) bytes += packed_stages * (kPairBN / 2) * 16 * h_bits;
+    bytes += 4 * 2 * kPairBN * (int)sizeof(float);
+    bytes += 512;
+    return bytes + 1024;
+}
+
+template <bool PART, int MODE>
+__global__ void __launch_bounds__(PART ? 192 + kUnpackThreads : 192, 1)
+contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                        const ContractionArgs p) {
+    using namespace sm100;
+    constexpr int BN = kPairBN;
+    constexpr int HALF = BN / 2;                              // rows of B held by this CTA
+    constexpr int STAGES = PART ? kPairStagesPart : kPairStagesFull;
+    constexpr int A_BYTES = a_stage_bytes();
+    constexpr int B_BYTES = b_stage_bytes(HALF);
+    constexpr uint32_t TMEM_COLS = 2 * BN;
+    constexpr uint32_t IDESC = idesc_i8(2 * kBM, BN);
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sA = smem;
+    uint8_t* sB = sA + STAGES * A_BYTES;
+    const int packed_bytes = PART ? HALF * 16 * p.h_bits : 0;
+    uint8_t* sP = sB + STAGES * B_BYTES;
+    float* sScale = reinterpret_cast<float*>(sP + (PART ? p.packed_stages * packed_bytes : 0));   // [4 warps][BN]
+    float* sBias = sScale + 4 * BN;
+    uint64_t* full = reinterpret_cast<uint64_t*>(sBias + 4 * BN);
+    uint64_t* empty = full + STAGES;
+    uint64_t* pfull = empty + STAGES;
+    uint64_t* pempty = pfull + kMaxPackedStages;
+    uint64_t* tfull = pempty + kMaxPackedStages;
+    uint64_t* tempty = tfull + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();                  // 0 = leader
+    const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+    const int num_tiles = p.m_tiles * p.n_tiles;              // m_tiles counts 256-row tiles here
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(smem_u32(&full[s]), PART ? 1 + 2 * kUnpackGroupWarps : 1);   // + one unpack group in each CTA
+            mbar_init(smem_u32(&empty[s]), 1);
+        }
+        for (int s = 0; s < kMaxPackedStages; ++s) {
+            mbar_init(smem_u32(&pfull[s]), 1);
+            mbar_init(smem_u32(&pempty[s]), kUnpackGroupWarps);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&tfull[b]), 1);
+            mbar_init(smem_u32(&tempty[b]), 8);                // four epilogue warps in each CTA
+        }
+        *abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&tmA);
+        prefetch_tensormap(&tmB);
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync_all();                                        // both CTAs' barriers exist before anyone signals across
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (both CTAs)
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+                int mt2, nt;
+                tile_coords(tile, p.m_tiles, p.n_tiles, mt2, nt);
+                const int mt = mt2 * 2 + (int)rank;            // this CTA's 128-row tile
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                    const uint32_t s = it % STAGES, use = it / STAGES;
+                    if (!(ok = mbar_wait_cluster(smem_u32(&empty[s]), (use & 1) ^ 1, abort_flag, p.status, 0x110u))) break;
+                    const uint32_t fb = map_to_cta(smem_u32(&full[s]), 0);        // the leader's barrier
+                    int n_sub = 1;
+                    if (MODE == kModeConv64) n_sub = min(2, p.g.taps - 2 * kb);
+                    const uint32_t a_bytes = (MODE == kModeConv64) ? n_sub * (A_BYTES / 2) : A_BYTES;
+                    const uint32_t b_bytes = PART ? 0u : ((MODE == kModeConv64) ? n_sub * (B_BYTES / 2) : B_BYTES);
+                    if (rank == 0) mbar_arrive_expect_tx(smem_u32(&full[s]), 2 * (a_bytes + b_bytes));
+                    if (MODE == kModeGemm) {
+                        tma_load_2d_pair(smem_u32(sA + s * A_BYTES), &tmA, kb * kBK, mt * kBM, fb);
+                    } else {
+                        const TileOrigin o = conv_tile_origin(p.g, mt);
+                        for (int sub = 0; sub < n_sub; ++sub) {
+                            const int tap = (MODE == kModeConv64) ? 2 * kb + sub : kb / p.g.cblocks;
+                            const int c0 = (MODE == kModeConv64) ? 0 : (kb % p.g.cblocks) * 128;
+                            const int r = tap / p.g.S, sx = tap - r * p.g.S;
+                            tma_load_4d_pair(smem_u32(sA + s * A_BYTES + sub * (A_BYTES / 2)), &tmA, c0,
+                                             o.q0 * p.g.stride - p.g.pad + sx, o.p0 * p.g.stride - p.g.pad + r, o.b0, fb);
+                        }
+                    }
+                    const int brow = nt * BN + (int)rank * HALF;                   // this CTA's half of the B tile
+                    if (PART) {
+                        // the packed tiles have a ring and a producer lane of their own (below)
+                    } else if (MODE == kModeConv64) {
+                        for (int sub = 0; sub < n_sub; ++sub)
+                            tma_load_2d_pair(smem_u32(sB + s * B_BYTES + sub * (B_BYTES / 2)), &tmB, kb * kBK + sub * 64, brow, fb);
+                    } else {
+                        tma_load_2d_pair(smem_u32(sB + s * B_BYTES), &tmB, kb * kBK, brow, fb);
+                    }
+                }
+            }
+            if (!ok) {
+                const long long t0 = clock64();                // let copies in flight land before shared memory is released
+                while (clock64() - t0 < (1ll << 22)) { }
+            }
+        } else if (PART && lane == 1) {
+            // ---- packed-tile producer: runs ahead of the A loads by up to the depth of its own ring, which
+            //      is what hides the latency of fetching the weights
+            uint32_t pit = 0;
+            bool ok = true;
+            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+                int mt2, nt;
+                tile_coords(tile, p.m_tiles, p.n_tiles, mt2, nt);
+                const int brow = nt * BN + (int)rank * HALF;
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++pit) {
+                    const uint32_t ps = pit % p.packed_stages, puse = pit / p.packed_stages;
+                    if (!(ok = mbar_wait(smem_u32(&pempty[ps]), (puse & 1) ^ 1, abort_flag, p.status, 0x111u))) break;
+                    const uint32_t pb = smem_u32(&pfull[ps]);
+                    mbar_arrive_expect_tx(pb, packed_bytes);
+                    tma_load_2d(smem_u32(sP + ps * packed_bytes), &tmB, kb * 16 * p.h_bits, brow, pb);
+                }
+            }
+            if (!ok) {
+                const long long t0 = clock64();
+                while (clock64() - t0 < (1ll << 22)) { }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (leader only)
+        if (lane == 0 && rank == 0) {
+            uint32_t it = 0, tl = 0;
+            bool ok = true;
+            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs, ++tl) {
+                const uint32_t buf = tl & 1, buse = tl >> 1;
+                if (!(ok = mbar_wait_cluster(smem_u32(&tempty[buf]), (buse & 1) ^ 1, abort_flag, p.status, 0x120u))) break;
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + buf * BN;
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                    const uint32_t s = it % STAGES, use = it / STAGES;
+                    if (!(ok = mbar_wait_cluster(smem_u32(&full[s]), use & 1, abort_flag, p.status, 0x121u))) break;
+                    tc_fence_after_sync();
+                    if (MODE == kModeConv64) {
+                        const int n_sub = min(2, p.g.taps - 2 * kb);
+                        for (int sub = 0; sub < n_sub; ++sub) {
+                            const uint64_t da = smem_desc_sw64(smem_u32(sA + s * A_BYTES + sub * (A_BYTES / 2)));
+                            const uint64_t db = smem_desc_sw64(smem_u32(sB + s * B_BYTES + sub * (B_BYTES / 2)));
+#pragma unroll
+                            for (int k = 0; k < 2; ++k)
+                                mma_i8_pair(d_tmem, da + 2 * k, db + 2 * k, IDESC, (kb | sub | k) != 0);
+                        }
+                    } else {
+                        const uint64_t da = smem_desc_sw128(smem_u32(sA + s * A_BYTES));
+                        const uint64_t db = smem_desc_sw128(smem_u32(sB + s * B_BYTES));
+#pragma unroll
+                        for (int k = 0; k < kBK / 32; ++k)
+                            mma_i8_pair(d_tmem, da + 2 * k, db + 2 * k, IDESC, (kb | k) != 0);
+                    }
+                    mma_commit_pair(smem_u32(&empty[s]));      // frees the stage in both CTAs
+                }
+                if (ok) mma_commit_pair(smem_u32(&tfull[buf]));
+            }
+        }
+    } else if (warp < 6) {
+        // ------------------------------------------------------------------ epilogue (both CTAs, own 128 rows)
+        const int quarter = warp & 3;
+        uint32_t tl = 0;
+        bool ok = true;
+        const bool vec_f32 = (p.y != nullptr) && !p.y_is_bf16 && ((p.ldy & 3) == 0) &&
+                             ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
+        const bool vec_bf16 = (p.y != nullptr) && p.y_is_bf16 && ((p.ldy & 7) == 0) &&
+                              ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
+        const bool vec_acc = (p.acc_out != nullptr) && ((p.ld_acc & 3) == 0) &&
+                             ((reinterpret_cast<uintptr_t>(p.acc_out) & 15) == 0);
+        float* sc_w = sScale + (warp - 2) * BN;
+        float* bs_w = sBias + (warp - 2) * BN;
+        for (int tile = pair; ok && tile < num_tiles; tile += num_pairs, ++tl) {
+            int mt2, nt;
+            tile_coords(tile, p.m_tiles, p.n_tiles, mt2, nt);
+            const int mt = mt2 * 2 + (int)rank;
+            const uint32_t buf = tl & 1, buse = tl >> 1;
+            const int n0 = nt * BN;
+            __syncwarp();
+            for (int j = lane; j < BN; j += 32) {
+                const int col = n0 + j;
+                float sc = 0.f, bs = 0.f;
+                if (col < p.N) {
+                    sc = __fmul_rn(__fmul_rn(__fmul_rn(p.act_scale, p.w_scale[col]), p.pow2_l), p.unshift);
+                    if (p.bias) bs = p.bias[col];
+                }
+                sc_w[j] = sc;
+                bs_w[j] = bs;
+            }
+            __syncwarp();
+            ok = mbar_wait_cluster(smem_u32(&tfull[buf]), buse & 1, abort_flag, p.status, 0x130u);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after_sync();
+            long long row;
+            bool row_ok;
+            if (MODE == kModeGemm) {
+                row = (long long)mt * kBM + quarter * 32 + lane;
+                row_ok = row < p.M;
+            } else {
+                const TileOrigin o = conv_tile_origin(p.g, mt);
+                const int ml = quarter * 32 + lane;
+                const int qq = o.q0 + (ml & ((1 << p.g.tw_log2) - 1));
+                const int pp = o.p0 + ((ml >> p.g.tw_log2) & ((1 << p.g.th_log2) - 1));
+                const int bb = o.b0 + (ml >> (p.g.tw_log2 + p.g.th_log2));
+                row_ok = qq < p.g.Wo && pp < p.g.Ho && bb < p.g.B;
+                row = ((long long)bb * p.g.Ho + pp) * p.g.Wo + qq;
+            }
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld_32x32(tmem_base + buf * BN + c * 32 + ((uint32_t)(quarter * 32) << 16), r);
+                tmem_ld_wait();
+                const int col0 = n0 + c * 32;
+                if (!row_ok || col0 >= p.N) continue;
+                store_chunk(p, row, col0, r, sc_w + c * 32, bs_w + c * 32, vec_acc, vec_f32, vec_bf16);
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&tempty[buf]), 0));
+        }
+    } else if (PART) {
+        // ------------------------------------------------------------------ unpackers (both CTAs, own half of B)
+        const int group = (warp - 6) / kUnpackGroupWarps;
+        const int utid = (threadIdx.x - 192) % kUnpackGroupThreads;
+        uint32_t it = 0;
+        bool ok = true;
+        for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+            for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                if ((int)(it % kUnpackGroups) != group) continue;
+                const uint32_t s = it % STAGES, use = it / STAGES;
+                const uint32_t ps = it % p.packed_stages, puse = it / p.packed_stages;
+                ok = mbar_wait(smem_u32(&pfull[ps]), puse & 1, abort_flag, p.status, 0x140u) &&
+                     mbar_wait_cluster(smem_u32(&empty[s]), (use & 1) ^ 1, abort_flag, p.status, 0x141u);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const uint8_t* src = sP + ps * packed_bytes;
+                uint8_t* dst = sB + s * B_BYTES;
+                switch (p.h_bits) {
+                    case 1: unpack_tile<HALF, MODE, 1, kUnpackGroupThreads>(src, dst, utid); break;
+                    case 2: unpack_tile<HALF, MODE, 2, kUnpackGroupThreads>(src, dst, utid); break;
+                    case 3: unpack_tile<HALF, MODE, 3, kUnpackGroupThreads>(src, dst, utid); break;
+                    case 4: unpack_tile<HALF, MODE, 4, kUnpackGroupThreads>(src, dst, utid); break;
+                    case 5: unpack_tile<HALF, MODE, 5, kUnpackGroupThreads>(src, dst, utid); break;
+                    case 6: unpack_tile<HALF, MODE, 6, kUnpackGroupThreads>(src, dst, utid); break;
+                    default: unpack_tile<HALF, MODE, 7, kUnpackGroupThreads>(src, dst, utid); break;
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive_cluster(map_to_cta(smem_u32(&full[s]), 0));
+                    mbar_arrive(smem_u32(&pempty[ps]));
+                }
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync_all();          // the partner's shared memory and TMEM stay alive until both CTAs are done
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc_pair(tmem_base, TMEM_COLS);
+    }
+}
+
+}  // namespace nq

@@ -4,7 +4,9 @@
 #include <stdint.h>
 
 #include "../../include/nq.h"
-#include "nq_contraction.cuh"
+#include <stdlib.h>
+
+#include "nq_contraction_pair.cuh"
 #include "nq_internal.cuh"
 
 namespace nq {
@@ -63,7 +65,7 @@ namespace {
 
 template <int BN, bool PART, int MODE>
 int launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const ContractionArgs& a, cudaStream_t stream) {
-    const int smem = contraction_smem_bytes(BN, PART, a.h_bits);
+    const int smem = contraction_smem_bytes(BN, PART, a.h_bits, a.packed_stages);
     static int configured[64] = {0};       // largest opt-in done so far, per device, for this instantiation
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return NQ_ERR_CUDA;
@@ -86,6 +88,58 @@ int launch_mode(int mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const 
     return launch<BN, PART, kModeGemm>(tmA, tmB, a, s);
 }
 
+// CTA-pair kernel: a cluster of two CTAs per 256 x 256 tile
+template <bool PART, int MODE>
+int launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const ContractionArgs& a, cudaStream_t stream) {
+    const int smem = pair_smem_bytes(PART, a.h_bits, a.packed_stages);
+    static int configured[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return NQ_ERR_CUDA;
+    if (smem > configured[dev]) {
+        if (cudaFuncSetAttribute(contraction_pair_kernel<PART, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 smem) != cudaSuccess)
+            return NQ_ERR_CUDA;
+        configured[dev] = smem;
+    }
+    const int tiles = a.m_tiles * a.n_tiles;
+    const int max_pairs = sm_count() / 2;
+    const int pairs = tiles < max_pairs ? tiles : max_pairs;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * pairs, 1, 1);
+    cfg.blockDim = dim3(PART ? 192 + kUnpackThreads : 192, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, contraction_pair_kernel<PART, MODE>, tmA, tmB, a) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return NQ_ERR_CUDA;
+    }
+    return NQ_OK;
+}
+
+template <bool PART>
+int launch_pair_mode(int mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const ContractionArgs& a, cudaStream_t s) {
+    if (mode == kModeConv128) return launch_pair<PART, kModeConv128>(tmA, tmB, a, s);
+    if (mode == kModeConv64) return launch_pair<PART, kModeConv64>(tmA, tmB, a, s);
+    return launch_pair<PART, kModeGemm>(tmA, tmB, a, s);
+}
+
+// NQ_SINGLE_CTA=1 in the environment keeps every contraction on the one-CTA-per-tile kernel (for comparisons)
+bool pairs_enabled() {
+    static int cached = -1;
+    if (cached < 0) {
+        const char* e = getenv("NQ_SINGLE_CTA");
+        cached = (e && e[0] == '1') ? 0 : 1;
+    }
+    return cached == 1;
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 }  // namespace
@@ -98,10 +152,13 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
                     const float* w_scale, float act_scale, const float* bias, int64_t M, int64_t N, int64_t K,
                     int32_t* acc_out, int64_t ld_acc, void* Y, int64_t ldy, int y_dtype, cudaStream_t stream) {
     const int bn = N > 128 ? 256 : (N > 64 ? 128 : 64);
+    // wide outputs with at least two 128-row tiles run on CTA pairs (256 x 256 tiles, half of B per CTA)
+    const bool pair = bn == kPairBN && m_tiles >= 2 && pairs_enabled();
+    const int b_box_rows = pair ? kPairBN / 2 : bn;
     ContractionArgs a{};
     if (geom) a.g = *geom;
     a.M = (int)M; a.N = (int)N; a.K = (int)K;
-    a.m_tiles = m_tiles;
+    a.m_tiles = pair ? (m_tiles + 1) / 2 : m_tiles;
     a.n_tiles = (int)((N + bn - 1) / bn);
     a.k_blocks = k_blocks;
     a.w_scale = w_scale; a.bias = bias; a.act_scale = act_scale;
@@ -115,16 +172,27 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
         a.acc_shift = 8 - h_bits;
         a.unshift = 1.0f / (float)(1 << a.acc_shift);
         a.h_bits = h_bits;
+        // as deep a ring of packed tiles as shared memory allows: it is what hides the load latency of B
+        // (pair kernel: a multiple of its unpack group count, see nq_contraction_pair.cuh)
+        a.packed_stages = 0;
+        const int step = pair ? kUnpackGroups : 1;
+        for (int d = kMaxPackedStages; d >= step; d -= step)
+            if ((pair ? pair_smem_bytes(true, h_bits, d) : contraction_smem_bytes(bn, true, h_bits, d)) <= kSmemLimit) {
+                a.packed_stages = d;
+                break;
+            }
+        if (a.packed_stages == 0) return NQ_ERR_UNSUPPORTED;
         const uint64_t row_bytes = (uint64_t)((K + 127) / 128) * 16 * h_bits;
-        int st = encode_tensor_map_2d(&tmB, Bmat, row_bytes, (uint64_t)N, row_bytes, 16 * h_bits, bn, 0);
+        int st = encode_tensor_map_2d(&tmB, Bmat, row_bytes, (uint64_t)N, row_bytes, 16 * h_bits, b_box_rows, 0);
         if (st != NQ_OK) return st;
     } else {
         a.pow2_l = 1.0f; a.unshift = 1.0f; a.acc_shift = 0; a.h_bits = 0;
         int st = (mode == kModeConv64)
-                     ? encode_tensor_map_2d(&tmB, Bmat, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, 64, bn, 64)
-                     : encode_tensor_map_2d(&tmB, Bmat, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, kBK, bn, 128);
+                     ? encode_tensor_map_2d(&tmB, Bmat, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, 64, b_box_rows, 64)
+                     : encode_tensor_map_2d(&tmB, Bmat, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, kBK, b_box_rows, 128);
         if (st != NQ_OK) return st;
     }
+    if (pair) return part ? launch_pair_mode<true>(mode, tmA, tmB, a, stream) : launch_pair_mode<false>(mode, tmA, tmB, a, stream);
     if (part) {
         if (bn == 256) return launch_mode<256, true>(mode, tmA, tmB, a, stream);
         if (bn == 128) return launch_mode<128, true>(mode, tmA, tmB, a, stream);
