@@ -11,8 +11,10 @@
 // issuer (only in the even, "leader" CTA; it also owns the TMEM allocation in both), warps 2-5 epilogue,
 // warps 6-13 unpackers (part-bit).  Barrier protocol, all barriers at the same offsets in both CTAs:
 //   full[s]    lives in the leader: 1 arrival by the leader's producer, which announces the bytes of BOTH
-//              CTAs' loads; the partner's loads complete on it through its cluster address; in part-bit
-//              mode the unpack warps of both CTAs arrive on it too
+//              CTAs' loads; the partner's loads complete on it through its cluster address.  In part-bit
+//              mode the leader's unpack warps arrive on it, and each of the partner's unpack warps sends it
+//              4 announced bytes with an asynchronous remote store (a cluster-scope release arrival costs
+//              the issuing warp over a thousand cycles; measured)
 //   empty[s]   one per CTA, arrived on in both CTAs at once by the leader's tcgen05.commit
 //   tfull[b]   likewise (accumulator b complete)
 //   tempty[b]  lives in the leader: the epilogue warps of both CTAs arrive (8 arrivals)
@@ -31,7 +33,10 @@ constexpr int kPairStagesPart = 4;
 // on the leader's barrier across the cluster) of different stages overlap.  Ring depths are multiples of the
 // group count, so that a ring slot is always served by the same group, in order: a parity wait is only valid
 // for a waiter that is at most one phase behind.
-constexpr int kUnpackGroups = 4;
+#ifndef NQ_UNPACK_GROUPS
+#define NQ_UNPACK_GROUPS 4
+#endif
+constexpr int kUnpackGroups = NQ_UNPACK_GROUPS;
 constexpr int kUnpackGroupWarps = kUnpackWarps / kUnpackGroups;
 constexpr int kUnpackGroupThreads = kUnpackGroupWarps * 32;
 static_assert(kPairStagesPart % kUnpackGroups == 0, "a stage slot must belong to one unpack group");
@@ -74,6 +79,7 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     uint64_t* tempty = tfull + 2;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    uint32_t* signal_sink = tmem_slot + 2;                    // landing place of the partner's signal stores
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -83,7 +89,7 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(smem_u32(&full[s]), PART ? 1 + 2 * kUnpackGroupWarps : 1);   // + one unpack group in each CTA
+            mbar_init(smem_u32(&full[s]), PART ? 1 + kUnpackGroupWarps : 1);   // + the leader's unpack group
             mbar_init(smem_u32(&empty[s]), 1);
         }
         for (int s = 0; s < kMaxPackedStages; ++s) {
@@ -126,7 +132,8 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                     if (MODE == kModeConv64) n_sub = min(2, p.g.taps - 2 * kb);
                     const uint32_t a_bytes = (MODE == kModeConv64) ? n_sub * (A_BYTES / 2) : A_BYTES;
                     const uint32_t b_bytes = PART ? 0u : ((MODE == kModeConv64) ? n_sub * (B_BYTES / 2) : B_BYTES);
-                    if (rank == 0) mbar_arrive_expect_tx(smem_u32(&full[s]), 2 * (a_bytes + b_bytes));
+                    // (part-bit: + 4 bytes from each warp of the partner's unpack group)
+                    if (rank == 0) mbar_arrive_expect_tx(smem_u32(&full[s]), 2 * (a_bytes + b_bytes) + (PART ? 4 * kUnpackGroupWarps : 0));
                     if (MODE == kModeGemm) {
                         tma_load_2d_pair(smem_u32(sA + s * A_BYTES), &tmA, kb * kBK, mt * kBM, fb);
                     } else {
@@ -302,7 +309,8 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive_cluster(map_to_cta(smem_u32(&full[s]), 0));
+                    if (rank == 0) mbar_arrive(smem_u32(&full[s]));
+                    else signal_remote_tx4(map_to_cta(smem_u32(signal_sink), 0), map_to_cta(smem_u32(&full[s]), 0));
                     mbar_arrive(smem_u32(&pempty[ps]));
                 }
             }

@@ -175,6 +175,14 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// Fire-and-forget signal to a barrier in another CTA of the cluster: an asynchronous 4-byte store to `sink`
+// there that counts 4 bytes on `bar` when it lands (both are cluster addresses).  Ordered after the issuing
+// thread's earlier generic-proxy writes by a preceding fence.proxy.async; unlike a cluster-scope release
+// arrival it does not stall the issuing warp.
+__device__ __forceinline__ void signal_remote_tx4(uint32_t cluster_sink, uint32_t cluster_bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
+                 ::"r"(cluster_sink), "r"(0u), "r"(cluster_bar) : "memory");
+}
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
