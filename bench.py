@@ -269,7 +269,7 @@ def run_ours(args, rank, world, local_rank):
     int8_peak = 2.0 * peaks["bf16_tflops"]
     achieved = gemm_ops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
     roofline = {
-        "bound": "tensor", "kernel": "contraction_kernel (tcgen05 kind::i8): every GEMM launch of the timed steps",
+        "bound": "tensor", "kernel": "contraction_pair_kernel / contraction_kernel (tcgen05 kind::i8): every GEMM launch of the timed steps",
         "achieved": round(achieved, 1), "peak": round(int8_peak, 1), "unit": "TOP/s",
         "frac": round(achieved / int8_peak, 4),
         "peak_source": "2 x the %s bf16 burst figure (dense INT8 : bf16 nominal ratio 4.5 : 2.25)" % peaks["source"],
