@@ -26,8 +26,12 @@ namespace nq {
 
 constexpr int kBM = 128;           // tile rows (M) = TMEM lanes
 constexpr int kBK = 128;           // K bytes per stage = one 128-byte swizzle row
-constexpr int kStagesFull = 4;
-constexpr int kStagesPart = 3;
+// Ring depth by tile width: narrow tiles have small stages and little work per stage, so they need more of
+// them in flight to cover the load latency (full-bit 8 / 6 / 4 stages of 24 / 32 / 48 KB; part-bit leaves
+// room for the packed ring).
+__host__ __device__ constexpr int stages_for(int bn, bool part) {
+    return part ? (bn == 64 ? 6 : bn == 128 ? 4 : 3) : (bn == 64 ? 8 : bn == 128 ? 6 : 4);
+}
 constexpr int kMaxPackedStages = 8;     // ring of packed (still INTh) B tiles; the depth in use is chosen by the host
 constexpr int kGroupM = 16;        // tile rasterisation: 16 M-tiles share a band of N-tiles
 
@@ -73,7 +77,7 @@ __host__ __device__ constexpr int b_stage_bytes(int bn) { return bn * kBK; }
 constexpr int kSmemLimit = 227 * 1024;   // dynamic shared memory a block may opt in to
 
 __host__ __device__ inline int contraction_smem_bytes(int bn, bool part, int h_bits, int packed_stages) {
-    int stages = part ? kStagesPart : kStagesFull;
+    int stages = stages_for(bn, part);
     int bytes = stages * (a_stage_bytes() + b_stage_bytes(bn));
     if (part) bytes += packed_stages * bn * 16 * h_bits;
     bytes += 4 * 2 * bn * (int)sizeof(float);   // scale and bias, one private copy per epilogue warp
@@ -260,7 +264,7 @@ __global__ void __launch_bounds__(PART ? 192 + kUnpackThreads : 192, 1)
 contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                    const ContractionArgs p) {
     using namespace sm100;
-    constexpr int STAGES = PART ? kStagesPart : kStagesFull;
+    constexpr int STAGES = stages_for(BN, PART);
     constexpr int A_BYTES = a_stage_bytes();
     constexpr int B_BYTES = b_stage_bytes(BN);
     constexpr uint32_t TMEM_COLS = (2 * BN < 32) ? 32 : 2 * BN;       // power of two >= 32

@@ -90,6 +90,55 @@ __global__ void __launch_bounds__(256) im2col_kernel(const int8_t* __restrict__ 
     *reinterpret_cast<uint4*>(a + m * ld + k0) = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
+// The same patch matrix for layers with few input channels (the stem): one block per output row (b, p).  The
+// R input rows it needs are staged in shared memory for all channels with the padding columns already
+// zero, and a small table gives, for every k, where its byte sits relative to the patch origin; each output
+// byte is then two shared-memory reads, and whole 16-byte chunks go out coalesced.
+__global__ void __launch_bounds__(256) im2col_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ a,
+                                                          nq_conv_desc d, int Ho, int Wo, int K, int ld) {
+    extern __shared__ uint8_t sm[];
+    const int Wp = d.W + 2 * d.pad;
+    uint8_t* patch = sm;                                           // [R][Cin][Wp]
+    uint16_t* lut = reinterpret_cast<uint16_t*>(sm + ((d.R * d.Cin * Wp + 15) & ~15));   // [ld]
+    const int p = blockIdx.x, b = blockIdx.y;
+    for (int i = threadIdx.x; i < d.R * d.Cin * Wp; i += blockDim.x) {
+        const int col = i % Wp, rc = i / Wp;
+        const int ci = rc % d.Cin, r = rc / d.Cin;
+        const int ih = p * d.stride - d.pad + r, iw = col - d.pad;
+        uint8_t v = 0;
+        if (ih >= 0 && ih < d.H && iw >= 0 && iw < d.W) {
+            const size_t off = d.x_nchw ? (((size_t)b * d.Cin + ci) * d.H + ih) * d.W + iw
+                                        : (((size_t)b * d.H + ih) * d.W + iw) * d.Cin + ci;
+            v = (uint8_t)x[off];
+        }
+        patch[i] = v;
+    }
+    for (int k = threadIdx.x; k < ld; k += blockDim.x) {
+        uint16_t o = 0xffffu;                                      // beyond K: zero
+        if (k < K) {
+            const int tap = k / d.Cin, ci = k - tap * d.Cin;
+            const int r = tap / d.S, s = tap - r * d.S;
+            o = (uint16_t)((r * d.Cin + ci) * Wp + s);
+        }
+        lut[k] = o;
+    }
+    __syncthreads();
+    const int cpr = ld / 16;
+    int8_t* out = a + ((size_t)b * Ho + p) * Wo * ld;
+    for (int idx = threadIdx.x; idx < Wo * cpr; idx += blockDim.x) {
+        const int q = idx / cpr, k0 = (idx - q * cpr) * 16;
+        const int base = q * d.stride;
+        uint32_t w[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const uint32_t o = lut[k0 + j];
+            const uint32_t v = (o == 0xffffu) ? 0u : patch[o + base];
+            w[j >> 2] |= v << (8 * (j & 3));
+        }
+        *reinterpret_cast<uint4*>(out + (size_t)q * ld + k0) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
 bool implicit_ok(const nq_conv_desc& d) { return d.Cin == 64 || (d.Cin > 0 && d.Cin % 128 == 0); }
 
 bool desc_ok(const nq_conv_desc* d) {
@@ -149,7 +198,13 @@ int nq_conv_implicit_gemm(const int8_t* X, const void* Wt, int64_t ldw, int part
         // explicit patch matrix, then the plain GEMM path
         const int ld = (int)((K + 15) / 16 * 16);
         const long long chunks = M * (ld / 16);
-        im2col_kernel<<<(unsigned)((chunks + 255) / 256), 256, 0, stream>>>(X, (int8_t*)workspace, *d, Ho, Wo, (int)K, ld, chunks);
+        const size_t rows_smem = (((size_t)d->R * d->Cin * (d->W + 2 * d->pad) + 15) & ~size_t(15)) + (size_t)ld * 2;
+        if (rows_smem <= 48 * 1024 && (size_t)d->R * d->Cin * (d->W + 2 * d->pad) + (size_t)Wo * d->stride < 0xffff &&
+            Ho <= 65535 * 32 && d->B <= 65535) {
+            im2col_rows_kernel<<<dim3(Ho, d->B), 256, rows_smem, stream>>>(X, (int8_t*)workspace, *d, Ho, Wo, (int)K, ld);
+        } else {
+            im2col_kernel<<<(unsigned)((chunks + 255) / 256), 256, 0, stream>>>(X, (int8_t*)workspace, *d, Ho, Wo, (int)K, ld, chunks);
+        }
         if (cudaGetLastError() != cudaSuccess) return NQ_ERR_CUDA;
         int st = encode_tensor_map_2d(&tmA, workspace, (uint64_t)K, (uint64_t)M, (uint64_t)ld, kBK, kBM, 128);
         if (st != NQ_OK) return st;

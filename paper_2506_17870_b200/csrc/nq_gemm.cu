@@ -151,9 +151,30 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
                     const void* Bmat, int64_t ldb, bool part, int n_bits, int h_bits,
                     const float* w_scale, float act_scale, const float* bias, int64_t M, int64_t N, int64_t K,
                     int32_t* acc_out, int64_t ld_acc, void* Y, int64_t ldy, int y_dtype, cudaStream_t stream) {
-    const int bn = N > 128 ? 256 : (N > 64 ? 128 : 64);
-    // wide outputs with at least two 128-row tiles run on CTA pairs (256 x 256 tiles, half of B per CTA)
-    const bool pair = bn == kPairBN && m_tiles >= 2 && pairs_enabled();
+    // Tile shape: the widest tile reuses operands best, but a small problem must first of all fill the
+    // machine.  Estimate, for each candidate, (waves of tiles over the SMs) x (stages per tile) x (cycles per
+    // stage, measured orders of magnitude: narrow tiles are load-bound, the wide single-CTA tile is
+    // shared-memory-bound) and take the cheapest.
+    const int sms = sm_count();
+    int bn = 64;
+    bool pair = false;
+    {
+        double best = 1e300;
+        const int cand_bn[4] = {64, 128, 256, 256};
+        const bool cand_pair[4] = {false, false, false, true};
+        const double stage_cycles[4] = {260.0, 330.0, 800.0, 560.0};
+        for (int c = 0; c < 4; ++c) {
+            if (cand_pair[c] && (!pairs_enabled() || m_tiles < 2)) continue;
+            if (c > 0 && N <= cand_bn[c - 1] && !(c == 3)) continue;          // no wider than the output needs
+            if (c == 3 && N <= 128) continue;
+            const long long nt = (N + cand_bn[c] - 1) / cand_bn[c];
+            const long long tiles = (cand_pair[c] ? (m_tiles + 1) / 2 : m_tiles) * nt;
+            const long long slots = cand_pair[c] ? sms / 2 : sms;
+            const double waves = (double)((tiles + slots - 1) / slots);
+            const double cost = waves * (k_blocks * stage_cycles[c] + 2500.0);   // + per-tile epilogue / fill
+            if (cost < best) { best = cost; bn = cand_bn[c]; pair = cand_pair[c]; }
+        }
+    }
     const int b_box_rows = pair ? kPairBN / 2 : bn;
     ContractionArgs a{};
     if (geom) a.g = *geom;
