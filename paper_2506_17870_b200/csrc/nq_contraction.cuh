@@ -8,9 +8,9 @@
 //               INTh tile in part-bit mode) into a ring of shared-memory stages
 //   warp 1      MMA issuer: one thread issues four tcgen05.mma kind::i8 (K = 32 each) per stage into
 //               a TMEM accumulator; owns the TMEM allocation
-//   warps 2-5   epilogue: tcgen05.ld the accumulator (each warp its 32-lane quarter), scale, store.
+//   warps 2-9   epilogue: tcgen05.ld the accumulator (each warp a 32-lane quarter and half of the columns), scale, store.
 //               Two accumulators alternate so the epilogue of tile i overlaps the MMAs of tile i+1
-//   warps 6-13  (part-bit only) unpackers: expand packed INTh fields into the swizzled int8 B tile.
+//   warps 10-17 (part-bit only) unpackers: expand packed INTh fields into the swizzled int8 B tile.
 //               The field goes to the TOP h bits of the byte, i.e. the byte is w_high * 2^(8-h); the
 //               accumulator is then 2^(8-h) times too large, exactly, and the epilogue takes it out
 //               (arithmetic shift for the int32 output, an exact power-of-two factor in the scale).
@@ -70,6 +70,18 @@ struct ContractionArgs {
     unsigned int* status;
 };
 
+// Thread layout of a block: warp 0 producer, warp 1 MMA issuer, then the epilogue warps, then (part-bit) the
+// unpack warps.  Eight epilogue warps: two per TMEM lane quarter, each taking half of the tile's columns -- a
+// single warp per scheduler cannot hide the latency of its own convert-and-store chain (measured: the
+// epilogue, not the stores, capped output-bound problems at 1.3 TB/s with four warps).
+constexpr int kEpiWarps = 8;
+constexpr int kFirstUnpackWarp = 2 + kEpiWarps;
+constexpr int kBaseThreads = (2 + kEpiWarps) * 32;
+// Output staging of one epilogue warp: 32 rows x 64 bytes, rows 80 bytes apart (an odd multiple of 16 keeps
+// the row-wise writes free of bank conflicts).
+constexpr int kEpiRowPitch = 80;
+constexpr int kEpiStageBytes = 32 * kEpiRowPitch;
+
 __host__ __device__ constexpr int a_stage_bytes() { return kBM * kBK; }
 __host__ __device__ constexpr int b_stage_bytes(int bn) { return bn * kBK; }
 
@@ -80,7 +92,8 @@ __host__ __device__ inline int contraction_smem_bytes(int bn, bool part, int h_b
     int stages = stages_for(bn, part);
     int bytes = stages * (a_stage_bytes() + b_stage_bytes(bn));
     if (part) bytes += packed_stages * bn * 16 * h_bits;
-    bytes += 4 * 2 * bn * (int)sizeof(float);   // scale and bias, one private copy per epilogue warp
+    bytes += 4 * 2 * bn * (int)sizeof(float);   // scale and bias: each epilogue warp keeps those of its half of the columns
+    bytes += kEpiWarps * kEpiStageBytes;        // output staging, one per epilogue warp
     bytes += 512;                       // barriers, TMEM base, abort flag
     return bytes + 1024;                // slack to align the base to 1024 B
 }
@@ -259,8 +272,85 @@ __device__ __forceinline__ void store_chunk(const ContractionArgs& p, long long 
     }
 }
 
+// 64 bytes of each of the warp's 32 rows, written with coalesced stores.  In the accumulator a lane owns one ROW,
+// so storing from registers makes every store instruction touch 32 different cache lines with 16 bytes each,
+// and the load/store unit spends a cycle per line: on output-bound problems that, not HBM, set the pace.  Here
+// the warp lays the 32 x 64-byte block out in shared memory and reads it back with four consecutive lanes on
+// one row: every instruction then touches 8 lines with 64 contiguous bytes each.  `q` is the lane's own row,
+// `row` / `row_ok` its row index and validity; all 32 lanes must call.
+__device__ __forceinline__ void store_rows64(uint8_t* stage, int lane, const uint4 (&q)[4], int row, bool row_ok,
+                                             uint8_t* base, long long pitch_bytes, long long col_byte) {
+    uint4* mine = reinterpret_cast<uint4*>(stage + lane * kEpiRowPitch);
+    mine[0] = q[0]; mine[1] = q[1]; mine[2] = q[2]; mine[3] = q[3];
+    __syncwarp();
+#pragma unroll
+    for (int pass = 0; pass < 4; ++pass) {
+        const int rr = pass * 8 + (lane >> 2), cg = lane & 3;
+        const int grow = __shfl_sync(0xffffffffu, row, rr);
+        const bool ok = __shfl_sync(0xffffffffu, (int)row_ok, rr) != 0;
+        const uint4 v = *reinterpret_cast<const uint4*>(stage + rr * kEpiRowPitch + cg * 16);
+        if (ok) *reinterpret_cast<uint4*>(base + grow * pitch_bytes + col_byte + cg * 16) = v;
+    }
+    __syncwarp();
+}
+
+// The epilogue of one warp for 32 consecutive columns: same arithmetic as store_chunk, coalesced stores.
+__device__ __forceinline__ void store_chunk_warp(const ContractionArgs& p, int row, bool row_ok, int col0,
+                                                 const uint32_t (&r)[32], const float* sc, const float* bs,
+                                                 bool vec_acc, bool vec_f32, bool vec_bf16, uint8_t* stage, int lane) {
+    const bool full_chunk = col0 + 32 <= p.N;
+    const bool acc_fast = p.acc_out == nullptr || (full_chunk && vec_acc);
+    const bool y_fast = p.y == nullptr || (full_chunk && (p.y_is_bf16 ? vec_bf16 : vec_f32));
+    if (!acc_fast || !y_fast) {                        // ragged or unaligned: the plain per-row path
+        if (row_ok) store_chunk(p, row, col0, r, sc, bs, vec_acc, vec_f32, vec_bf16);
+        return;
+    }
+    uint4 q[4];
+    if (p.acc_out) {
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                q[j] = make_uint4((uint32_t)((int)r[half * 16 + 4 * j] >> p.acc_shift), (uint32_t)((int)r[half * 16 + 4 * j + 1] >> p.acc_shift),
+                                  (uint32_t)((int)r[half * 16 + 4 * j + 2] >> p.acc_shift), (uint32_t)((int)r[half * 16 + 4 * j + 3] >> p.acc_shift));
+            store_rows64(stage, lane, q, row, row_ok, reinterpret_cast<uint8_t*>(p.acc_out), p.ld_acc * 4,
+                         (long long)(col0 + half * 16) * 4);
+        }
+    }
+    if (p.y) {
+        float v[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            float t = __fmul_rn(__int2float_rn((int)r[j]), sc[j]);
+            v[j] = p.bias ? __fadd_rn(t, bs[j]) : t;
+        }
+        if (!p.y_is_bf16) {
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    q[j] = make_uint4(__float_as_uint(v[half * 16 + 4 * j]), __float_as_uint(v[half * 16 + 4 * j + 1]),
+                                      __float_as_uint(v[half * 16 + 4 * j + 2]), __float_as_uint(v[half * 16 + 4 * j + 3]));
+                store_rows64(stage, lane, q, row, row_ok, reinterpret_cast<uint8_t*>(p.y), p.ldy * 4,
+                             (long long)(col0 + half * 16) * 4);
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                __nv_bfloat162 a = __floats2bfloat162_rn(v[8 * j], v[8 * j + 1]);
+                __nv_bfloat162 b = __floats2bfloat162_rn(v[8 * j + 2], v[8 * j + 3]);
+                __nv_bfloat162 c2 = __floats2bfloat162_rn(v[8 * j + 4], v[8 * j + 5]);
+                __nv_bfloat162 d = __floats2bfloat162_rn(v[8 * j + 6], v[8 * j + 7]);
+                q[j] = make_uint4(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b),
+                                  *reinterpret_cast<uint32_t*>(&c2), *reinterpret_cast<uint32_t*>(&d));
+            }
+            store_rows64(stage, lane, q, row, row_ok, reinterpret_cast<uint8_t*>(p.y), p.ldy * 2, (long long)col0 * 2);
+        }
+    }
+}
+
 template <int BN, bool PART, int MODE>
-__global__ void __launch_bounds__(PART ? 192 + kUnpackThreads : 192, 1)
+__global__ void __launch_bounds__(PART ? kBaseThreads + kUnpackThreads : kBaseThreads, 1)
 contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                    const ContractionArgs p) {
     using namespace sm100;
@@ -278,7 +368,8 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     uint8_t* sP = sB + STAGES * B_BYTES;
     float* sScale = reinterpret_cast<float*>(sP + (PART ? p.packed_stages * packed_bytes : 0));   // [4 warps][BN]
     float* sBias = sScale + 4 * BN;                                                             // [4 warps][BN]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sBias + 4 * BN);
+    uint8_t* sStage = reinterpret_cast<uint8_t*>(sBias + 4 * BN);                               // [kEpiWarps][kEpiStageBytes]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sStage + kEpiWarps * kEpiStageBytes);
     // barrier map: full[STAGES], empty[STAGES], pfull[2], pempty[2], tfull[2], tempty[2]
     uint64_t* full = bars;
     uint64_t* empty = full + STAGES;
@@ -304,7 +395,7 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&tfull[b]), 1);
-            mbar_init(smem_u32(&tempty[b]), 4);                // one arrival per epilogue warp
+            mbar_init(smem_u32(&tempty[b]), kEpiWarps);        // one arrival per epilogue warp
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -421,9 +512,10 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 if (ok) mma_commit(smem_u32(&tfull[buf]));   // accumulator complete
             }
         }
-    } else if (warp < 6) {
+    } else if (warp < kFirstUnpackWarp) {
         // ------------------------------------------------------------------ epilogue
         const int quarter = warp & 3;                  // TMEM lanes this warp may read
+        const int chalf = (warp - 2) >> 2;             // which half of the tile's columns it handles
         uint32_t tl = 0;
         bool ok = true;
         const bool vec_f32 = (p.y != nullptr) && !p.y_is_bf16 && ((p.ldy & 3) == 0) &&
@@ -439,11 +531,11 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             const int n0 = nt * BN;
             // per-channel factor: fl(fl(act * w_scale) * 2^l), then the exact 2^-(8-h) of the unpack.
             // Each warp keeps a private copy, so the epilogue warps never wait on one another.
-            float* sc_w = sScale + (warp - 2) * BN;
-            float* bs_w = sBias + (warp - 2) * BN;
+            float* sc_w = sScale + (warp - 2) * (BN / 2);      // scales of this warp's half of the columns
+            float* bs_w = sBias + (warp - 2) * (BN / 2);
             __syncwarp();
-            for (int j = lane; j < BN; j += 32) {
-                const int col = n0 + j;
+            for (int j = lane; j < BN / 2; j += 32) {
+                const int col = n0 + chalf * (BN / 2) + j;
                 float sc = 0.f, bs = 0.f;
                 if (col < p.N) {
                     sc = __fmul_rn(__fmul_rn(__fmul_rn(p.act_scale, p.w_scale[col]), p.pow2_l), p.unshift);
@@ -472,22 +564,27 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 row_ok = qq < p.g.Wo && pp < p.g.Ho && bb < p.g.B;
                 row = ((long long)bb * p.g.Ho + pp) * p.g.Wo + qq;
             }
+            constexpr int CHUNKS = BN / 64;                // 32-column chunks per warp (half of the tile)
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
+            for (int cc = 0; cc < CHUNKS; ++cc) {
+                const int c = chalf * CHUNKS + cc;
                 uint32_t r[32];
                 tmem_ld_32x32(tmem_base + buf * BN + c * 32 + ((uint32_t)(quarter * 32) << 16), r);
                 tmem_ld_wait();
+                if (cc == CHUNKS - 1) {                    // last read of the accumulator: hand it back before storing
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&tempty[buf]));
+                }
                 const int col0 = n0 + c * 32;
-                if (!row_ok || col0 >= p.N) continue;
-                store_chunk(p, row, col0, r, sc_w + c * 32, bs_w + c * 32, vec_acc, vec_f32, vec_bf16);
+                if (col0 >= p.N) continue;
+                store_chunk_warp(p, (int)row, row_ok, col0, r, sc_w + cc * 32, bs_w + cc * 32, vec_acc, vec_f32, vec_bf16,
+                                 sStage + (warp - 2) * kEpiStageBytes, lane);
             }
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&tempty[buf]));
         }
     } else if (PART) {
         // ------------------------------------------------------------------ unpackers (warps 6-13)
-        const int utid = threadIdx.x - 192;
+        const int utid = threadIdx.x - kBaseThreads;
         uint32_t it = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {

@@ -8,8 +8,8 @@
 // half as many weights.
 //
 // Roles per CTA are those of the single-CTA kernel (nq_contraction.cuh): warp 0 TMA producer, warp 1 MMA
-// issuer (only in the even, "leader" CTA; it also owns the TMEM allocation in both), warps 2-5 epilogue,
-// warps 6-13 unpackers (part-bit).  Barrier protocol, all barriers at the same offsets in both CTAs:
+// issuer (only in the even, "leader" CTA; it also owns the TMEM allocation in both), warps 2-9 epilogue,
+// warps 10-17 unpackers (part-bit).  Barrier protocol, all barriers at the same offsets in both CTAs:
 //   full[s]    lives in the leader: 1 arrival by the leader's producer, which announces the bytes of BOTH
 //              CTAs' loads; the partner's loads complete on it through its cluster address.  In part-bit
 //              mode the leader's unpack warps arrive on it, and each of the partner's unpack warps sends it
@@ -17,7 +17,7 @@
 //              the issuing warp over a thousand cycles; measured)
 //   empty[s]   one per CTA, arrived on in both CTAs at once by the leader's tcgen05.commit
 //   tfull[b]   likewise (accumulator b complete)
-//   tempty[b]  lives in the leader: the epilogue warps of both CTAs arrive (8 arrivals)
+//   tempty[b]  lives in the leader: its own epilogue warps arrive, the partner's send 4 announced bytes each
 //   pfull / pempty  packed-tile ring, private to each CTA
 // Every wait is bounded; every TMA load has a single destination CTA.
 #pragma once
@@ -46,12 +46,13 @@ __host__ __device__ inline int pair_smem_bytes(bool part, int h_bits, int packed
     int bytes = stages * (a_stage_bytes() + b_stage_bytes(kPairBN / 2));
     if (part) bytes += packed_stages * (kPairBN / 2) * 16 * h_bits;
     bytes += 4 * 2 * kPairBN * (int)sizeof(float);
+    bytes += kEpiWarps * kEpiStageBytes;
     bytes += 512;
     return bytes + 1024;
 }
 
 template <bool PART, int MODE>
-__global__ void __launch_bounds__(PART ? 192 + kUnpackThreads : 192, 1)
+__global__ void __launch_bounds__(PART ? kBaseThreads + kUnpackThreads : kBaseThreads, 1)
 contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                         const ContractionArgs p) {
     using namespace sm100;
@@ -71,7 +72,8 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     uint8_t* sP = sB + STAGES * B_BYTES;
     float* sScale = reinterpret_cast<float*>(sP + (PART ? p.packed_stages * packed_bytes : 0));   // [4 warps][BN]
     float* sBias = sScale + 4 * BN;
-    uint64_t* full = reinterpret_cast<uint64_t*>(sBias + 4 * BN);
+    uint8_t* sStage = reinterpret_cast<uint8_t*>(sBias + 4 * BN);
+    uint64_t* full = reinterpret_cast<uint64_t*>(sStage + kEpiWarps * kEpiStageBytes);
     uint64_t* empty = full + STAGES;
     uint64_t* pfull = empty + STAGES;
     uint64_t* pempty = pfull + kMaxPackedStages;
@@ -98,7 +100,8 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&tfull[b]), 1);
-            mbar_init(smem_u32(&tempty[b]), 8);                // four epilogue warps in each CTA
+            // the leader's epilogue warps arrive; the partner's send 4 bytes each, announced by the MMA thread
+            mbar_init(smem_u32(&tempty[b]), kEpiWarps + 1);
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -191,6 +194,8 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             for (int tile = pair; ok && tile < num_tiles; tile += num_pairs, ++tl) {
                 const uint32_t buf = tl & 1, buse = tl >> 1;
                 if (!(ok = mbar_wait_cluster(smem_u32(&tempty[buf]), (buse & 1) ^ 1, abort_flag, p.status, 0x120u))) break;
+                // this use's hand-back: the leader's warps arrive, the partner's warps each send 4 bytes
+                mbar_arrive_expect_tx(smem_u32(&tempty[buf]), 4 * kEpiWarps);
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * BN;
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
@@ -218,9 +223,10 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 if (ok) mma_commit_pair(smem_u32(&tfull[buf]));
             }
         }
-    } else if (warp < 6) {
+    } else if (warp < kFirstUnpackWarp) {
         // ------------------------------------------------------------------ epilogue (both CTAs, own 128 rows)
         const int quarter = warp & 3;
+        const int chalf = (warp - 2) >> 2;             // which half of the tile's columns this warp handles
         uint32_t tl = 0;
         bool ok = true;
         const bool vec_f32 = (p.y != nullptr) && !p.y_is_bf16 && ((p.ldy & 3) == 0) &&
@@ -229,8 +235,8 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                               ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
         const bool vec_acc = (p.acc_out != nullptr) && ((p.ld_acc & 3) == 0) &&
                              ((reinterpret_cast<uintptr_t>(p.acc_out) & 15) == 0);
-        float* sc_w = sScale + (warp - 2) * BN;
-        float* bs_w = sBias + (warp - 2) * BN;
+        float* sc_w = sScale + (warp - 2) * (BN / 2);      // scales of this warp's half of the columns
+        float* bs_w = sBias + (warp - 2) * (BN / 2);
         for (int tile = pair; ok && tile < num_tiles; tile += num_pairs, ++tl) {
             int mt2, nt;
             tile_coords(tile, p.m_tiles, p.n_tiles, mt2, nt);
@@ -238,8 +244,8 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             const uint32_t buf = tl & 1, buse = tl >> 1;
             const int n0 = nt * BN;
             __syncwarp();
-            for (int j = lane; j < BN; j += 32) {
-                const int col = n0 + j;
+            for (int j = lane; j < BN / 2; j += 32) {
+                const int col = n0 + chalf * (BN / 2) + j;
                 float sc = 0.f, bs = 0.f;
                 if (col < p.N) {
                     sc = __fmul_rn(__fmul_rn(__fmul_rn(p.act_scale, p.w_scale[col]), p.pow2_l), p.unshift);
@@ -267,23 +273,31 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 row_ok = qq < p.g.Wo && pp < p.g.Ho && bb < p.g.B;
                 row = ((long long)bb * p.g.Ho + pp) * p.g.Wo + qq;
             }
+            constexpr int CHUNKS = BN / 64;                // 32-column chunks per warp (half of the tile)
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
+            for (int cc = 0; cc < CHUNKS; ++cc) {
+                const int c = chalf * CHUNKS + cc;
                 uint32_t r[32];
                 tmem_ld_32x32(tmem_base + buf * BN + c * 32 + ((uint32_t)(quarter * 32) << 16), r);
                 tmem_ld_wait();
+                if (cc == CHUNKS - 1) {                    // last read of the accumulator: hand it back before storing
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (rank == 0) mbar_arrive(smem_u32(&tempty[buf]));
+                        else signal_remote_tx4(map_to_cta(smem_u32(signal_sink), 0), map_to_cta(smem_u32(&tempty[buf]), 0));
+                    }
+                }
                 const int col0 = n0 + c * 32;
-                if (!row_ok || col0 >= p.N) continue;
-                store_chunk(p, row, col0, r, sc_w + c * 32, bs_w + c * 32, vec_acc, vec_f32, vec_bf16);
+                if (col0 >= p.N) continue;
+                store_chunk_warp(p, (int)row, row_ok, col0, r, sc_w + cc * 32, bs_w + cc * 32, vec_acc, vec_f32, vec_bf16,
+                                 sStage + (warp - 2) * kEpiStageBytes, lane);
             }
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(&tempty[buf]), 0));
         }
     } else if (PART) {
         // ------------------------------------------------------------------ unpackers (both CTAs, own half of B)
-        const int group = (warp - 6) / kUnpackGroupWarps;
-        const int utid = (threadIdx.x - 192) % kUnpackGroupThreads;
+        const int group = (warp - kFirstUnpackWarp) / kUnpackGroupWarps;
+        const int utid = (threadIdx.x - kBaseThreads) % kUnpackGroupThreads;
         uint32_t it = 0;
         bool ok = true;
         for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {

@@ -77,7 +77,7 @@ int launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const ContractionArgs
     }
     const int tiles = a.m_tiles * a.n_tiles;
     const int grid = tiles < sm_count() ? tiles : sm_count();
-    contraction_kernel<BN, PART, MODE><<<grid, PART ? 192 + kUnpackThreads : 192, smem, stream>>>(tmA, tmB, a);
+    contraction_kernel<BN, PART, MODE><<<grid, PART ? kBaseThreads + kUnpackThreads : kBaseThreads, smem, stream>>>(tmA, tmB, a);
     return cudaGetLastError() == cudaSuccess ? NQ_OK : NQ_ERR_CUDA;
 }
 
@@ -106,7 +106,7 @@ int launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const Contractio
     const int pairs = tiles < max_pairs ? tiles : max_pairs;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * pairs, 1, 1);
-    cfg.blockDim = dim3(PART ? 192 + kUnpackThreads : 192, 1, 1);
+    cfg.blockDim = dim3(PART ? kBaseThreads + kUnpackThreads : kBaseThreads, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
