@@ -6,7 +6,10 @@ One "step" is one pass of the whole path over the large square GEMM sweep (M = N
 
     decompose -> drop-low (page-out) -> recompose (page-in) -> part-bit GEMM,   plus one full-bit GEMM per size,
 
-followed by a pass over ResNet-18-shaped convolution layers (implicit GEMM, both modes).
+followed by the ResNet-18-shaped convolution stack (config 2: 20 convolutions + classifier, batch 32, NCHW
+int8 activations, implicit GEMM, both modes).  After the timed steps the whole-model page-out / page-in of a
+ResNet-101-shaped and a ViT-B-shaped model (one batched launch each, cold L2) is timed separately and
+reported under rows.model_switch.
 `value` is the integer-op throughput of the whole step (2*M*N*K per contraction; the codec kernels
 add time but no ops) in TOPS, summed over ranks.  Per-row numbers (TOPS per mode, GB/s per codec
 kernel) are reported under "rows".
@@ -38,7 +41,6 @@ N_BITS = 8
 ACT_SCALE = 0.05
 METRIC = "nested_int8_gemm_tops"
 CONV_H = 6
-CONV_LAYER_NAMES = ("l1b0c1", "l2b0c1", "l2b0c2", "l2b0ds", "l3b0c2", "l4b0c2")
 
 
 def measured_peaks():
@@ -113,8 +115,9 @@ def make_host_inputs(sizes):
 
 
 def conv_bench_layers():
+    """Config 2: the whole ResNet-18-shaped stack, 20 convolutions + the classifier."""
     from paper_2506_17870_b200 import workloads as wl
-    return [l for l in wl.resnet18_layers() if l.name in CONV_LAYER_NAMES]
+    return wl.resnet18_layers()
 
 
 def _conv_available(nq, torch, dev):
@@ -247,6 +250,7 @@ def run_ours(args, rank, world, local_rank):
     gpu_launches = launches[0]
 
     e2e = _run_e2e(nq, torch, sizes, host, state, args, world)
+    model_switch = _model_switch(nq, torch, wl, dev) if (rank == 0 and args.model_switch) else None
 
     if world > 1:
         t = torch.tensor([total_ms, e2e["ms_per_step"]], device=dev, dtype=torch.float64)
@@ -275,8 +279,8 @@ def run_ours(args, rank, world, local_rank):
         "peak_source": "2 x the %s bf16 burst figure (dense INT8 : bf16 nominal ratio 4.5 : 2.25)" % peaks["source"],
         "launches": gemm_n, "avg_launch_ms": round(gemm_ms / max(gemm_n, 1), 4), "traffic": None,
     }
-    conv_note = (", + %d ResNet-18-shaped conv layers, batch %d, both modes" % (len(conv_layers), args.conv_batch)
-                 if have_conv else "")
+    conv_note = (", + config 2: the ResNet-18-shaped stack (%d layers), batch %d, NCHW int8 in, both modes"
+                 % (len(conv_layers), args.conv_batch) if have_conv else "")
     line = {
         "metric": METRIC, "value": round(value, 2), "unit": "TOPS", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak",
@@ -293,6 +297,8 @@ def run_ours(args, rank, world, local_rank):
                 "ms_per_step": round(e2e["ms_per_step"], 3), "covers": "the GEMM sweep (codec + both GEMM modes)"},
         "roofline": roofline, "rows": rows,
     }
+    if model_switch is not None:
+        line["rows"]["model_switch"] = model_switch
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(sizes, host, args.cpu_rows)
     return line
@@ -320,11 +326,67 @@ def _summarise_rows(events, conv_layers, conv_batch, peaks):
             M, N, K = L.gemm_view(conv_batch)
             t = 2.0 * M * N * K / (ms * 1e-3) / 1e12
             out.setdefault(kind, {})[s] = {"tops": round(t, 1), "ms": round(ms, 4), "gemm_view": [M, N, K]}
+    for kind in ("conv_full", "conv_part"):
+        if kind in out:
+            tot_ms = sum(v["ms"] for v in out[kind].values())
+            tot_ops = sum(2.0 * v["gemm_view"][0] * v["gemm_view"][1] * v["gemm_view"][2] for v in out[kind].values())
+            out[kind + "_stack"] = {"ms": round(tot_ms, 4), "tops": round(tot_ops / (tot_ms * 1e-3) / 1e12, 1),
+                                    "layers": len(out[kind])}
     for (kind, s), vals in agg.items():
         g = float(np.mean(vals))
         out["codec"].setdefault(kind, {})[str(s)] = {"gbs": round(g, 0), "frac_hbm": round(g / hbm, 3)}
     out["codec"]["algorithmic_bytes_per_weight"] = codec_bytes
     out["peaks"] = {"int8_tops": int8_peak, "hbm_gbs": hbm, "source": peaks["source"]}
+    return out
+
+
+def _model_switch(nq, torch, wl, dev):
+    """Whole-model page-out and page-in as one batched launch each, INT(8|6) ResNet-101 (105 tensors) and INT(8|4)
+    ViT-B/16 blocks (48 tensors).  Three copies of each model are rotated so that every launch finds its data in
+    HBM, not in the 126 MB L2; CUDA events around three back-to-back launches (one per copy), median of 12."""
+    peaks = measured_peaks()
+    out = {}
+    models = {
+        "resnet101_int8_6": (6, [(L.Cout, L.K) for L in wl.resnet101_layers()]),
+        "vit_b16_int8_4": (4, [(n, k) for _, k, n in wl.vit_b16_linears()]),
+    }
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(wl.BASE_SEED)
+    for name, (h, shapes) in models.items():
+        copies = []
+        for c in range(3):
+            tensors = []
+            for rows, cols in shapes:
+                ld = -(-cols // 16) * 16
+                w = torch.randint(-128, 128, (rows, ld), dtype=torch.int8, device=dev, generator=gen)[:, :cols]
+                m = torch.randint(0, 2, (rows, ld), dtype=torch.uint8, device=dev, generator=gen)[:, :cols]
+                hi, lo = nq.nq_decompose(w, m, N_BITS, h, True)
+                tensors.append({"w_int": w, "packed_high": hi, "packed_low": lo})
+            copies.append(nq.nq_batch_plan(tensors))
+        weights = sum(r * c for r, c in shapes)
+        nbytes = weights * 2.125
+        res = {}
+        for kind, fn in (("page_out", nq.nq_drop_low_batched), ("page_in", nq.nq_recompose_batched)):
+            for i in range(3):
+                fn(copies[i], N_BITS, h, True)
+            torch.cuda.synchronize()
+            ts = []
+            for i in range(12):                       # one launch per copy inside each event pair
+                a = torch.cuda.Event(enable_timing=True)
+                b = torch.cuda.Event(enable_timing=True)
+                a.record()
+                for c in range(3):
+                    fn(copies[c], N_BITS, h, True)
+                b.record()
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b) / 3)
+            ms = float(np.median(ts))
+            gbs = nbytes / (ms * 1e-3) / 1e9
+            res[kind] = {"us": round(ms * 1e3, 1), "gbs": round(gbs, 0), "frac_hbm": round(gbs / peaks["hbm_gbs"], 3)}
+        res["weights"] = weights
+        res["tensors"] = len(shapes)
+        res["algorithmic_mb"] = round(nbytes / 1e6, 1)
+        out[name] = res
     return out
 
 
@@ -437,6 +499,7 @@ def main():
     ap.add_argument("--conv-batch", type=int, default=32)
     ap.add_argument("--no-conv", dest="conv", action="store_false")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-model-switch", dest="model_switch", action="store_false")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))

@@ -113,9 +113,10 @@ NQ_API int nq_pack(const int8_t *values, int64_t ld, int bits, int64_t rows, int
  * Whole-model page-in / page-out in ONE launch.  A model is a list of tensors; the caller builds
  * the list once with nq_batch_plan and then switches the model with a single call.
  *   descs (host)   count entries
- *   table (device) at least nq_batch_table_bytes(count) bytes, 16-byte aligned; filled by
- *                  nq_batch_plan with a copy queued on `stream`
- *   total_units    work-item count nq_batch_plan reports; pass it back to the batched calls
+ *   table (device) at least nq_batch_table_bytes(descs, count) bytes, 16-byte aligned; filled by
+ *                  nq_batch_plan with a copy queued on `stream`.  It lists the tensors and cuts the model
+ *                  into work items (one thread block each) that never straddle two tensors.
+ *   work_items     the number of work items nq_batch_plan reports; pass it back to the batched calls
  * Every tensor of a batch shares (n_bits, h_bits, compensate).  w_int must be 16-byte aligned with
  * ld a multiple of 16 for every tensor of a batch (NQ_ERR_ALIGNMENT otherwise).
  */
@@ -126,12 +127,12 @@ typedef struct {
     int8_t *w_int;            /* (device) */
 } nq_tensor_desc;
 
-NQ_API int64_t nq_batch_table_bytes(int count);
+NQ_API int64_t nq_batch_table_bytes(const nq_tensor_desc *descs, int count);
 NQ_API int nq_batch_plan(const nq_tensor_desc *descs, int count, void *table, int64_t table_bytes,
-                  int64_t *total_units_out, void *stream);
-NQ_API int nq_recompose_batched(const void *table, int count, int64_t total_units,
+                  int64_t *work_items_out, void *stream);
+NQ_API int nq_recompose_batched(const void *table, int count, int64_t work_items,
                          int n_bits, int h_bits, int compensate, void *stream);
-NQ_API int nq_drop_low_batched(const void *table, int count, int64_t total_units,
+NQ_API int nq_drop_low_batched(const void *table, int count, int64_t work_items,
                         int n_bits, int h_bits, int compensate, void *stream);
 
 /*

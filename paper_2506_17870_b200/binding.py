@@ -185,7 +185,7 @@ def nq_pack(values: torch.Tensor, bits: int) -> torch.Tensor:
 
 
 class BatchPlan:
-    """Device table of a model's tensors (nq_batch_plan) plus the unit total the batched calls need."""
+    """Device table of a model's tensors (nq_batch_plan) plus the work-item count the batched calls need."""
 
     def __init__(self, table: torch.Tensor, count: int, total_units: int, keep: Sequence[torch.Tensor]):
         self.table, self.count, self.total_units, self._keep = table, count, total_units, list(keep)
@@ -205,7 +205,7 @@ def nq_batch_plan(tensors: Sequence[dict]) -> BatchPlan:
         arr[i] = nq_tensor_desc(w.shape[0], w.shape[1], _ld(w), t["packed_high"].data_ptr(),
                                 t["packed_low"].data_ptr(), w.data_ptr())
         keep += [w, t["packed_high"], t["packed_low"]]
-    nbytes = int(lib().nq_batch_table_bytes(count))
+    nbytes = int(lib().nq_batch_table_bytes(arr, count))
     table = torch.empty(nbytes, dtype=torch.uint8, device=device)
     total = ctypes.c_int64(0)
     _check(lib().nq_batch_plan(arr, count, _ptr(table), _i64(nbytes), ctypes.byref(total), _stream()), "nq_batch_plan")

@@ -392,23 +392,29 @@ struct BatchEntry {
 };
 static_assert(sizeof(BatchEntry) == 64, "table entry is 64 bytes");
 
+// A model is cut into work items of at most kItemUnits units, none of which straddles two tensors; block b of
+// the batched launch takes item b, so no thread ever searches the tensor table.
+#ifndef NQ_ITEM_UNITS
+#define NQ_ITEM_UNITS 1024
+#endif
+constexpr int kItemUnits = NQ_ITEM_UNITS;
+struct BatchItem {
+    int32_t entry;          // which tensor
+    int32_t units;          // how many units of it (<= kItemUnits)
+    int64_t first_unit;     // first unit inside that tensor
+};
+static_assert(sizeof(BatchItem) == 16, "work item is 16 bytes");
+
 template <int OP, class NestT>
-__global__ void __launch_bounds__(256, 4) codec_batched_kernel(const BatchEntry* __restrict__ table, int count,
-                                                               int64_t total_units, int n, int h, int comp) {
+__global__ void __launch_bounds__(256, 4) codec_batched_kernel(const BatchEntry* __restrict__ table,
+                                                               const BatchItem* __restrict__ items, int n, int h, int comp) {
     const NestT N(n, h, comp);
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < total_units; u += stride) {
-        int lo = 0, hi = count - 1;                 // last entry whose first_unit <= u
-        while (lo < hi) {
-            int mid = (lo + hi + 1) >> 1;
-            if (__ldg(&table[mid].first_unit) <= u) lo = mid; else hi = mid - 1;
-        }
-        const BatchEntry* e = table + lo;
-        TensorView t;
-        t.rows = __ldg(&e->rows); t.cols = __ldg(&e->cols); t.ld = __ldg(&e->ld);
-        t.hi = e->hi; t.lo = e->lo; t.w = e->w; t.mask = nullptr;
-        do_unit<OP>(t, u - __ldg(&e->first_unit), N, 0);
-    }
+    const BatchItem item = items[blockIdx.x];
+    const BatchEntry* e = table + item.entry;
+    TensorView t;
+    t.rows = __ldg(&e->rows); t.cols = __ldg(&e->cols); t.ld = __ldg(&e->ld);
+    t.hi = e->hi; t.lo = e->lo; t.w = e->w; t.mask = nullptr;
+    for (int i = threadIdx.x; i < item.units; i += blockDim.x) do_unit<OP>(t, item.first_unit + i, N, 0);
 }
 
 inline int launch_blocks(int64_t total_units) {
@@ -426,8 +432,9 @@ void launch_one(const TensorView& t, int64_t total, int n, int h, int comp, int 
     codec_kernel<OP, NestT><<<launch_blocks(total), 256, 0, s>>>(t, total, n, h, comp, bits);
 }
 template <int OP, class NestT>
-void launch_batch(const BatchEntry* table, int count, int64_t total, int n, int h, int comp, cudaStream_t s) {
-    codec_batched_kernel<OP, NestT><<<launch_blocks(total), 256, 0, s>>>(table, count, total, n, h, comp);
+void launch_batch(const BatchEntry* table, int count, int64_t items, int n, int h, int comp, cudaStream_t s) {
+    const BatchItem* list = reinterpret_cast<const BatchItem*>(table + count);
+    codec_batched_kernel<OP, NestT><<<(unsigned)items, 256, 0, s>>>(table, list, n, h, comp);
 }
 
 template <int OP, int H>
@@ -542,42 +549,63 @@ int nq_pack(const int8_t* values, int64_t ld, int bits, int64_t rows, int64_t co
     return run_single<OP_PACK>(t, 8, 4, 1, bits, stream);
 }
 
-int64_t nq_batch_table_bytes(int count) {
-    if (count < 0) return -1;
-    return (int64_t)(count > 0 ? count : 1) * (int64_t)sizeof(BatchEntry);
+static int64_t items_of(const nq_tensor_desc& d) {
+    const int64_t units = d.rows * ((d.cols + 127) / 128) * 4;
+    return (units + kItemUnits - 1) / kItemUnits;
+}
+
+int64_t nq_batch_table_bytes(const nq_tensor_desc* descs, int count) {
+    if (count < 0 || (count > 0 && !descs)) return -1;
+    int64_t items = 0;
+    for (int i = 0; i < count; ++i) {
+        if (descs[i].rows < 0 || descs[i].cols < 0) return -1;
+        items += items_of(descs[i]);
+    }
+    return (int64_t)(count > 0 ? count : 1) * (int64_t)sizeof(BatchEntry) + (items > 0 ? items : 1) * (int64_t)sizeof(BatchItem);
 }
 
 int nq_batch_plan(const nq_tensor_desc* descs, int count, void* table, int64_t table_bytes,
-                  int64_t* total_units_out, void* stream) {
-    if (count < 0 || (count > 0 && !descs) || !table || !total_units_out) return NQ_ERR_INVALID_ARG;
-    if (table_bytes < nq_batch_table_bytes(count)) return NQ_ERR_WORKSPACE;
+                  int64_t* work_items_out, void* stream) {
+    if (count < 0 || (count > 0 && !descs) || !table || !work_items_out) return NQ_ERR_INVALID_ARG;
+    const int64_t need = nq_batch_table_bytes(descs, count);
+    if (need < 0) return NQ_ERR_INVALID_ARG;
+    if (table_bytes < need) return NQ_ERR_WORKSPACE;
     if (!aligned16(table)) return NQ_ERR_ALIGNMENT;
-    std::vector<BatchEntry> host((size_t)count);
-    int64_t units = 0;
+    std::vector<unsigned char> host((size_t)need, 0);
+    BatchEntry* entries = reinterpret_cast<BatchEntry*>(host.data());
+    BatchItem* items = reinterpret_cast<BatchItem*>(host.data() + (size_t)count * sizeof(BatchEntry));
+    int64_t n_items = 0, units_before = 0;
     for (int i = 0; i < count; ++i) {
         const nq_tensor_desc& d = descs[i];
-        if (d.rows < 0 || d.cols < 0 || d.ld < d.cols) return NQ_ERR_INVALID_ARG;
+        if (d.ld < d.cols) return NQ_ERR_INVALID_ARG;
         if (d.rows > 0 && d.cols > 0) {
             if (!d.packed_high || !d.packed_low || !d.w_int) return NQ_ERR_INVALID_ARG;
             if (!aligned16(d.packed_high) || !aligned16(d.packed_low) || !aligned16(d.w_int) || (d.ld & 15))
                 return NQ_ERR_ALIGNMENT;
         }
-        BatchEntry& e = host[i];
+        BatchEntry& e = entries[i];
         e.rows = d.rows; e.cols = d.cols; e.ld = d.ld;
         e.hi = (uint8_t*)d.packed_high; e.lo = (uint8_t*)d.packed_low; e.w = d.w_int;
-        e.first_unit = units; e.pad_ = 0;
-        units += d.rows * ((d.cols + 127) / 128) * 4;
+        e.first_unit = units_before; e.pad_ = 0;
+        const int64_t units = d.rows * ((d.cols + 127) / 128) * 4;
+        units_before += units;
+        for (int64_t u = 0; u < units; u += kItemUnits) {
+            BatchItem& it = items[n_items++];
+            it.entry = i;
+            it.units = (int32_t)((units - u) < kItemUnits ? (units - u) : kItemUnits);
+            it.first_unit = u;
+        }
     }
-    *total_units_out = units;
-    if (count == 0) return NQ_OK;
+    *work_items_out = n_items;
+    if (count == 0 || n_items == 0) return NQ_OK;
     // the source is pageable host memory: the runtime stages it before this call returns
-    cudaError_t err = cudaMemcpyAsync(table, host.data(), (size_t)count * sizeof(BatchEntry),
+    cudaError_t err = cudaMemcpyAsync(table, host.data(), (size_t)count * sizeof(BatchEntry) + (size_t)n_items * sizeof(BatchItem),
                                       cudaMemcpyHostToDevice, (cudaStream_t)stream);
     return err == cudaSuccess ? NQ_OK : NQ_ERR_CUDA;
 }
 
 static int run_batched(int op, const void* table, int count, int64_t units, int n, int h, int comp, void* stream) {
-    if (count < 0 || units < 0 || !table) return NQ_ERR_INVALID_ARG;
+    if (count < 0 || units < 0 || units > 0x7fffffffLL || !table) return NQ_ERR_INVALID_ARG;
     if (!nest_ok(n, h)) return NQ_ERR_UNSUPPORTED;
     if (count == 0 || units == 0) return NQ_OK;
     const BatchEntry* entries = reinterpret_cast<const BatchEntry*>(table);
@@ -587,14 +615,14 @@ static int run_batched(int op, const void* table, int count, int64_t units, int 
     return cudaGetLastError() == cudaSuccess ? NQ_OK : NQ_ERR_CUDA;
 }
 
-int nq_recompose_batched(const void* table, int count, int64_t total_units, int n_bits, int h_bits, int compensate,
+int nq_recompose_batched(const void* table, int count, int64_t work_items, int n_bits, int h_bits, int compensate,
                          void* stream) {
-    return run_batched(OP_RECOMPOSE, table, count, total_units, n_bits, h_bits, compensate ? 1 : 0, stream);
+    return run_batched(OP_RECOMPOSE, table, count, work_items, n_bits, h_bits, compensate ? 1 : 0, stream);
 }
 
-int nq_drop_low_batched(const void* table, int count, int64_t total_units, int n_bits, int h_bits, int compensate,
+int nq_drop_low_batched(const void* table, int count, int64_t work_items, int n_bits, int h_bits, int compensate,
                         void* stream) {
-    return run_batched(OP_DROP_LOW, table, count, total_units, n_bits, h_bits, compensate ? 1 : 0, stream);
+    return run_batched(OP_DROP_LOW, table, count, work_items, n_bits, h_bits, compensate ? 1 : 0, stream);
 }
 
 }  // extern "C"
