@@ -230,11 +230,26 @@ __device__ __forceinline__ void store_chunk(const ContractionArgs& p, long long 
         }
     }
     if (p.y) {
+        // the 32 factors are the same for every lane: read them four at a time (a scalar read per column costs
+        // a shared-memory wavefront each, and the load/store data path is the busiest unit of this epilogue)
         float v[32];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            float t = __fmul_rn(__int2float_rn((int)r[j]), sc[j]);
-            v[j] = p.bias ? __fadd_rn(t, bs[j]) : t;
+        for (int j = 0; j < 32; j += 4) {
+            const float4 s4 = *reinterpret_cast<const float4*>(sc + j);
+            v[j] = __fmul_rn(__int2float_rn((int)r[j]), s4.x);
+            v[j + 1] = __fmul_rn(__int2float_rn((int)r[j + 1]), s4.y);
+            v[j + 2] = __fmul_rn(__int2float_rn((int)r[j + 2]), s4.z);
+            v[j + 3] = __fmul_rn(__int2float_rn((int)r[j + 3]), s4.w);
+        }
+        if (p.bias) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+                const float4 b4 = *reinterpret_cast<const float4*>(bs + j);
+                v[j] = __fadd_rn(v[j], b4.x);
+                v[j + 1] = __fadd_rn(v[j + 1], b4.y);
+                v[j + 2] = __fadd_rn(v[j + 2], b4.z);
+                v[j + 3] = __fadd_rn(v[j + 3], b4.w);
+            }
         }
         if (!p.y_is_bf16) {
             float* dst = reinterpret_cast<float*>(p.y) + row * p.ldy + col0;
@@ -318,11 +333,26 @@ __device__ __forceinline__ void store_chunk_warp(const ContractionArgs& p, int r
         }
     }
     if (p.y) {
+        // the 32 factors are the same for every lane: read them four at a time (a scalar read per column costs
+        // a shared-memory wavefront each, and the load/store data path is the busiest unit of this epilogue)
         float v[32];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            float t = __fmul_rn(__int2float_rn((int)r[j]), sc[j]);
-            v[j] = p.bias ? __fadd_rn(t, bs[j]) : t;
+        for (int j = 0; j < 32; j += 4) {
+            const float4 s4 = *reinterpret_cast<const float4*>(sc + j);
+            v[j] = __fmul_rn(__int2float_rn((int)r[j]), s4.x);
+            v[j + 1] = __fmul_rn(__int2float_rn((int)r[j + 1]), s4.y);
+            v[j + 2] = __fmul_rn(__int2float_rn((int)r[j + 2]), s4.z);
+            v[j + 3] = __fmul_rn(__int2float_rn((int)r[j + 3]), s4.w);
+        }
+        if (p.bias) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+                const float4 b4 = *reinterpret_cast<const float4*>(bs + j);
+                v[j] = __fadd_rn(v[j], b4.x);
+                v[j + 1] = __fadd_rn(v[j + 1], b4.y);
+                v[j + 2] = __fadd_rn(v[j + 2], b4.z);
+                v[j + 3] = __fadd_rn(v[j + 3], b4.w);
+            }
         }
         if (!p.y_is_bf16) {
 #pragma unroll
@@ -345,6 +375,23 @@ __device__ __forceinline__ void store_chunk_warp(const ContractionArgs& p, int r
                                   *reinterpret_cast<uint32_t*>(&c2), *reinterpret_cast<uint32_t*>(&d));
             }
             store_rows64(stage, lane, q, row, row_ok, reinterpret_cast<uint8_t*>(p.y), p.ldy * 2, (long long)col0 * 2);
+        }
+    }
+}
+
+// Per-channel output factors of 32 * PER_LANE consecutive columns starting at col_base, lane-strided:
+// fl(fl(act * w_scale) * 2^l), then the exact 2^-(8-h) that undoes the top-aligned unpack; and the bias.
+template <int PER_LANE>
+__device__ __forceinline__ void fetch_scales(const ContractionArgs& p, int col_base, int lane, float (&sc)[PER_LANE],
+                                             float (&bs)[PER_LANE]) {
+#pragma unroll
+    for (int i = 0; i < PER_LANE; ++i) {
+        const int col = col_base + lane + 32 * i;
+        sc[i] = 0.f;
+        bs[i] = 0.f;
+        if (col < p.N) {
+            sc[i] = __fmul_rn(__fmul_rn(__fmul_rn(p.act_scale, __ldg(p.w_scale + col)), p.pow2_l), p.unshift);
+            if (p.bias) bs[i] = __ldg(p.bias + col);
         }
     }
 }
@@ -516,6 +563,8 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         // ------------------------------------------------------------------ epilogue
         const int quarter = warp & 3;                  // TMEM lanes this warp may read
         const int chalf = (warp - 2) >> 2;             // which half of the tile's columns it handles
+        int staged_nt = -1;                            // column tile whose scales sit in shared memory
+        constexpr int SCALES_PER_LANE = BN / 64;       // a warp stages BN / 2 scales
         uint32_t tl = 0;
         bool ok = true;
         const bool vec_f32 = (p.y != nullptr) && !p.y_is_bf16 && ((p.ldy & 3) == 0) &&
@@ -534,17 +583,24 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             float* sc_w = sScale + (warp - 2) * (BN / 2);      // scales of this warp's half of the columns
             float* bs_w = sBias + (warp - 2) * (BN / 2);
             __syncwarp();
-            for (int j = lane; j < BN / 2; j += 32) {
-                const int col = n0 + chalf * (BN / 2) + j;
-                float sc = 0.f, bs = 0.f;
-                if (col < p.N) {
-                    sc = __fmul_rn(__fmul_rn(__fmul_rn(p.act_scale, p.w_scale[col]), p.pow2_l), p.unshift);
-                    if (p.bias) bs = p.bias[col];
-                }
-                sc_w[j] = sc;
-                bs_w[j] = bs;
+            if (nt != staged_nt) {                         // only the first tile: later ones are prefetched below
+                float sc_r[SCALES_PER_LANE], bs_r[SCALES_PER_LANE];
+                fetch_scales<SCALES_PER_LANE>(p, n0 + chalf * (BN / 2), lane, sc_r, bs_r);
+#pragma unroll
+                for (int i = 0; i < SCALES_PER_LANE; ++i) { sc_w[lane + 32 * i] = sc_r[i]; bs_w[lane + 32 * i] = bs_r[i]; }
+                staged_nt = nt;
             }
             __syncwarp();
+            // The next tile's scales are fetched now and land in registers while this tile is converted and
+            // stored; they go to shared memory at the end of the iteration.  (Fetched at the top of the next
+            // iteration instead, the global-memory round trip sat on every tile's critical path.)
+            int next_nt = -1;
+            float sc_n[SCALES_PER_LANE], bs_n[SCALES_PER_LANE];
+            if (tile + (int)gridDim.x < num_tiles) {
+                int mt_n;
+                tile_coords(tile + (int)gridDim.x, p.m_tiles, p.n_tiles, mt_n, next_nt);
+                if (next_nt != nt) fetch_scales<SCALES_PER_LANE>(p, next_nt * BN + chalf * (BN / 2), lane, sc_n, bs_n);
+            }
             ok = mbar_wait(smem_u32(&tfull[buf]), buse & 1, abort_flag, p.status, 0x30u);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -580,6 +636,12 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 if (col0 >= p.N) continue;
                 store_chunk_warp(p, (int)row, row_ok, col0, r, sc_w + cc * 32, bs_w + cc * 32, vec_acc, vec_f32, vec_bf16,
                                  sStage + (warp - 2) * kEpiStageBytes, lane);
+            }
+            if (next_nt >= 0 && next_nt != nt) {
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < SCALES_PER_LANE; ++i) { sc_w[lane + 32 * i] = sc_n[i]; bs_w[lane + 32 * i] = bs_n[i]; }
+                staged_nt = next_nt;
             }
         }
     } else if (PART) {

@@ -227,6 +227,8 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         // ------------------------------------------------------------------ epilogue (both CTAs, own 128 rows)
         const int quarter = warp & 3;
         const int chalf = (warp - 2) >> 2;             // which half of the tile's columns this warp handles
+        int staged_nt = -1;                            // column tile whose scales sit in shared memory
+        constexpr int SCALES_PER_LANE = BN / 64;       // a warp stages BN / 2 scales
         uint32_t tl = 0;
         bool ok = true;
         const bool vec_f32 = (p.y != nullptr) && !p.y_is_bf16 && ((p.ldy & 3) == 0) &&
@@ -244,17 +246,24 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             const uint32_t buf = tl & 1, buse = tl >> 1;
             const int n0 = nt * BN;
             __syncwarp();
-            for (int j = lane; j < BN / 2; j += 32) {
-                const int col = n0 + chalf * (BN / 2) + j;
-                float sc = 0.f, bs = 0.f;
-                if (col < p.N) {
-                    sc = __fmul_rn(__fmul_rn(__fmul_rn(p.act_scale, p.w_scale[col]), p.pow2_l), p.unshift);
-                    if (p.bias) bs = p.bias[col];
-                }
-                sc_w[j] = sc;
-                bs_w[j] = bs;
+            if (nt != staged_nt) {                         // only the first tile: later ones are prefetched below
+                float sc_r[SCALES_PER_LANE], bs_r[SCALES_PER_LANE];
+                fetch_scales<SCALES_PER_LANE>(p, n0 + chalf * (BN / 2), lane, sc_r, bs_r);
+#pragma unroll
+                for (int i = 0; i < SCALES_PER_LANE; ++i) { sc_w[lane + 32 * i] = sc_r[i]; bs_w[lane + 32 * i] = bs_r[i]; }
+                staged_nt = nt;
             }
             __syncwarp();
+            // The next tile's scales are fetched now and land in registers while this tile is converted and
+            // stored; they go to shared memory at the end of the iteration.  (Fetched at the top of the next
+            // iteration instead, the global-memory round trip sat on every tile's critical path.)
+            int next_nt = -1;
+            float sc_n[SCALES_PER_LANE], bs_n[SCALES_PER_LANE];
+            if (tile + num_pairs < num_tiles) {
+                int mt_n;
+                tile_coords(tile + num_pairs, p.m_tiles, p.n_tiles, mt_n, next_nt);
+                if (next_nt != nt) fetch_scales<SCALES_PER_LANE>(p, next_nt * BN + chalf * (BN / 2), lane, sc_n, bs_n);
+            }
             ok = mbar_wait_cluster(smem_u32(&tfull[buf]), buse & 1, abort_flag, p.status, 0x130u);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -292,6 +301,12 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 if (col0 >= p.N) continue;
                 store_chunk_warp(p, (int)row, row_ok, col0, r, sc_w + cc * 32, bs_w + cc * 32, vec_acc, vec_f32, vec_bf16,
                                  sStage + (warp - 2) * kEpiStageBytes, lane);
+            }
+            if (next_nt >= 0 && next_nt != nt) {
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < SCALES_PER_LANE; ++i) { sc_w[lane + 32 * i] = sc_n[i]; bs_w[lane + 32 * i] = bs_n[i]; }
+                staged_nt = next_nt;
             }
         }
     } else if (PART) {
