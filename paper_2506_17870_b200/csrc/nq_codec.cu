@@ -263,19 +263,19 @@ __device__ __forceinline__ void decompose_word(const NestT& N, uint32_t V, uint3
 template <class NestT>
 __device__ __forceinline__ uint32_t recompose_word(const NestT& N, uint32_t Thi, uint32_t Tlo) {
     uint32_t x = ((Thi >> (8 - N.n)) & N.mask_n) ^ N.bias;     // (w_high + 2^(h-1)) << l
-    uint32_t lo = (Tlo >> (8 - N.lb)) & N.mask_lb;
+    const uint32_t lo = Tlo >> (8 - N.lb);                      // low-aligned field; stray neighbour bits are masked below
     uint32_t a, s;
     if (N.comp) {          // l+1-bit field: low l bits drop in, the sign bit subtracts 2^l
         a = x | (lo & N.mask_l);
         s = lo & N.bit_l;
     } else {               // l-bit field: lo + 2^(l-1) drops in, then 2^(l-1) comes off
         uint32_t half = rep8(1u << (N.l - 1));
-        a = x | (lo ^ half);
+        a = x | ((lo & N.mask_l) ^ half);
         s = half;
     }
     // the only clip that can bind is the lower one (result below -2^(n-1)): an unsigned saturating subtract
     uint32_t wu = (N.comp && N.l == 7) ? subsat_u4(a, s) : subsat_small_u4(a, s);
-    return sub4(wu, N.bias);
+    return N.n == 8 ? (wu ^ H4) : sub4(wu, N.bias);             // back from the biased domain
 }
 
 // (w_int - w_low) / 2^l as an h-bit field
