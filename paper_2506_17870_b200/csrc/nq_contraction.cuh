@@ -62,6 +62,8 @@ struct ContractionArgs {
     int acc_shift;       // 8-h in part-bit mode, 0 otherwise
     int h_bits;          // part-bit: width of the packed field
     int packed_stages;   // part-bit: depth of the packed-tile ring (1..kMaxPackedStages)
+    const uint8_t* packed_b;   // part-bit: the packed matrix itself and its row pitch in bytes
+    long long packed_pitch;
     int32_t* acc_out;
     long long ld_acc;
     void* y;
@@ -156,6 +158,35 @@ __device__ __forceinline__ void expand_packed_unit(const PackedUnit& r, uint32_t
     }
 }
 
+// Write the 32 expanded bytes of one unit where the MMA expects them in the swizzled int8 tile of ROWS rows.
+template <int ROWS, int MODE>
+__device__ __forceinline__ void store_expanded_unit(uint8_t* __restrict__ dst, int row, int unit, const uint32_t (&T)[8]) {
+    if (MODE == kModeConv64) {
+        // two sub-tiles of 64-byte rows: units 0,1 feed the first, 2,3 the second; 64-byte swizzle
+        uint8_t* drow = dst + (unit >> 1) * (ROWS * 64) + row * 64;
+        const int sw = (row >> 1) & 3, c = (unit & 1) * 2;
+        *reinterpret_cast<uint4*>(drow + ((c ^ sw) << 4)) = make_uint4(T[0], T[1], T[2], T[3]);
+        *reinterpret_cast<uint4*>(drow + (((c + 1) ^ sw) << 4)) = make_uint4(T[4], T[5], T[6], T[7]);
+    } else {
+        uint8_t* drow = dst + row * 128;
+        const int sw = row & 7;
+        *reinterpret_cast<uint4*>(drow + (((2 * unit) ^ sw) << 4)) = make_uint4(T[0], T[1], T[2], T[3]);
+        *reinterpret_cast<uint4*>(drow + (((2 * unit + 1) ^ sw) << 4)) = make_uint4(T[4], T[5], T[6], T[7]);
+    }
+}
+
+// The same unit fetched straight from the packed matrix in global memory (group = start of the row's
+// 128-field group); a row past the end of the matrix reads as zeros.
+template <int H>
+__device__ __forceinline__ void fetch_packed_unit(const uint8_t* group, int unit, bool in_range, PackedUnit& r) {
+    r.a = make_uint4(0u, 0u, 0u, 0u); r.c = make_uint2(0u, 0u); r.d = 0u;
+    if (!in_range) return;
+    int off = 0;
+    if (H & 4) { r.a = sm100::ldg_stream_v4(group + unit * 16); off = 64; }
+    if (H & 2) { r.c = sm100::ldg_stream_v2(group + off + unit * 8); off += 32; }
+    if (H & 1) { r.d = sm100::ldg_stream_u32(group + off + unit * 4); }
+}
+
 constexpr int kUnpackWarps = 8;
 constexpr int kUnpackThreads = kUnpackWarps * 32;
 
@@ -180,18 +211,7 @@ __device__ __forceinline__ void unpack_tile(const uint8_t* __restrict__ src, uin
             const int row = task >> 2, unit = task & 3;
             uint32_t T[8];
             expand_packed_unit<H>(raw[i], T);
-            if (MODE == kModeConv64) {
-                // two sub-tiles of 64-byte rows: units 0,1 feed the first, 2,3 the second; 64-byte swizzle
-                uint8_t* drow = dst + (unit >> 1) * (ROWS * 64) + row * 64;
-                const int sw = (row >> 1) & 3, c = (unit & 1) * 2;
-                *reinterpret_cast<uint4*>(drow + ((c ^ sw) << 4)) = make_uint4(T[0], T[1], T[2], T[3]);
-                *reinterpret_cast<uint4*>(drow + (((c + 1) ^ sw) << 4)) = make_uint4(T[4], T[5], T[6], T[7]);
-            } else {
-                uint8_t* drow = dst + row * 128;
-                const int sw = row & 7;
-                *reinterpret_cast<uint4*>(drow + (((2 * unit) ^ sw) << 4)) = make_uint4(T[0], T[1], T[2], T[3]);
-                *reinterpret_cast<uint4*>(drow + (((2 * unit + 1) ^ sw) << 4)) = make_uint4(T[4], T[5], T[6], T[7]);
-            }
+            store_expanded_unit<ROWS, MODE>(dst, row, unit, T);
         }
     }
 }

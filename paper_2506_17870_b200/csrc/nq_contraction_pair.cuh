@@ -19,6 +19,14 @@
 //   tfull[b]   likewise (accumulator b complete)
 //   tempty[b]  lives in the leader: its own epilogue warps arrive, the partner's send 4 announced bytes each
 //   pfull / pempty  packed-tile ring, private to each CTA
+// DIRECT (part-bit, h <= 4): the packed fields never pass through shared memory; each unpack thread reads its
+// fields straight from the packed matrix into registers, one turn ahead of their use.  Reason, measured: the
+// shared-memory port carries per stage and SM 32 KB of operand reads, 16 KB of A, 16 KB of expanded B and the
+// packed tile twice (in by TMA, out to the unpack warps), 64 + 4h KB against 64 KB in the stage's 512 tensor
+// cycles, and the part-bit rate followed that sum (0.80 / 0.76 / 0.73 / 0.70 of the full-bit rate for h = 4 .. 7).
+// Direct reads lifted h = 4 from 2.40 to 2.93 POP/s at 8192^3; for h >= 5 the narrow slices need two or three
+// small loads per unit and the load/store unit becomes the limit instead (h = 7 fell to 1.7), so those keep the
+// ring.
 // Every wait is bounded; every TMA load has a single destination CTA.
 #pragma once
 #include "nq_contraction.cuh"
@@ -40,6 +48,7 @@ constexpr int kUnpackGroups = NQ_UNPACK_GROUPS;
 constexpr int kUnpackGroupWarps = kUnpackWarps / kUnpackGroups;
 constexpr int kUnpackGroupThreads = kUnpackGroupWarps * 32;
 static_assert(kPairStagesPart % kUnpackGroups == 0, "a stage slot must belong to one unpack group");
+constexpr int kPairUnitsPerThread = (kPairBN / 2) * 4 / kUnpackGroupThreads;   // 32-field units per stage and thread
 
 __host__ __device__ inline int pair_smem_bytes(bool part, int h_bits, int packed_stages) {
     const int stages = part ? kPairStagesPart : kPairStagesFull;
@@ -51,7 +60,80 @@ __host__ __device__ inline int pair_smem_bytes(bool part, int h_bits, int packed
     return bytes + 1024;
 }
 
-template <bool PART, int MODE>
+struct PairUnpackCtx {
+    uint8_t* sB;
+    uint64_t* full;
+    uint64_t* empty;
+    uint32_t* signal_sink;
+    volatile int* abort_flag;
+    uint32_t rank;
+    int pair, num_pairs, num_tiles, group, utid, lane;
+};
+
+// A group's position in the pair's sequence of K stages: iteration counter, tile and K block.
+struct StageCursor {
+    uint32_t it;
+    int tile, kb;
+};
+__device__ __forceinline__ void advance_cursor(StageCursor& c, int steps, int k_blocks, int num_pairs, int num_tiles) {
+    c.it += steps;
+    c.kb += steps;
+    while (c.kb >= k_blocks && c.tile < num_tiles) { c.kb -= k_blocks; c.tile += num_pairs; }
+}
+
+// The packed fields of one stage (this CTA's 128 rows of B x one 128-field group) into registers.
+template <int H>
+__device__ __forceinline__ void fetch_stage(const ContractionArgs& p, const PairUnpackCtx& cx, const StageCursor& c,
+                                            PackedUnit (&raw)[kPairUnitsPerThread]) {
+    int mt2, nt;
+    tile_coords(c.tile, p.m_tiles, p.n_tiles, mt2, nt);
+    const int brow = nt * kPairBN + (int)cx.rank * (kPairBN / 2);
+    const uint8_t* base = p.packed_b + (long long)c.kb * (16 * H);
+#pragma unroll
+    for (int i = 0; i < kPairUnitsPerThread; ++i) {
+        const int task = i * kUnpackGroupThreads + cx.utid;
+        const int row = brow + (task >> 2);
+        fetch_packed_unit<H>(base + (long long)row * p.packed_pitch, task & 3, row < p.N, raw[i]);
+    }
+}
+
+// One unpack group of the DIRECT variant: for each of its stages wait for the slot, expand the fields fetched a
+// turn earlier into the int8 tile, tell the leader's MMA thread, and only then fetch the fields of its next
+// stage -- they have until the group's next turn to arrive.  (Fetching before the proxy fence was slower.)
+template <int MODE, int H>
+__device__ __forceinline__ void pair_unpack_direct(const ContractionArgs& p, const PairUnpackCtx& cx) {
+    using namespace sm100;
+    constexpr int HALF = kPairBN / 2;
+    constexpr int B_BYTES = b_stage_bytes(HALF);
+    PackedUnit raw[kPairUnitsPerThread];
+    StageCursor cur{0u, cx.pair, 0};
+    advance_cursor(cur, cx.group, p.k_blocks, cx.num_pairs, cx.num_tiles);
+    if (cur.tile < cx.num_tiles) fetch_stage<H>(p, cx, cur, raw);
+    while (cur.tile < cx.num_tiles) {
+        const uint32_t s = cur.it % kPairStagesPart, use = cur.it / kPairStagesPart;
+        bool ok = mbar_wait_cluster(smem_u32(&cx.empty[s]), (use & 1) ^ 1, cx.abort_flag, p.status, 0x141u);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        uint8_t* dst = cx.sB + s * B_BYTES;
+#pragma unroll
+        for (int i = 0; i < kPairUnitsPerThread; ++i) {
+            const int task = i * kUnpackGroupThreads + cx.utid;
+            uint32_t T[8];
+            expand_packed_unit<H>(raw[i], T);
+            store_expanded_unit<HALF, MODE>(dst, task >> 2, task & 3, T);
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (cx.lane == 0) {
+            if (cx.rank == 0) mbar_arrive(smem_u32(&cx.full[s]));
+            else signal_remote_tx4(map_to_cta(smem_u32(cx.signal_sink), 0), map_to_cta(smem_u32(&cx.full[s]), 0));
+        }
+        advance_cursor(cur, kUnpackGroups, p.k_blocks, cx.num_pairs, cx.num_tiles);
+        if (cur.tile < cx.num_tiles) fetch_stage<H>(p, cx, cur, raw);
+    }
+}
+
+template <bool PART, int MODE, bool DIRECT = false>
 __global__ void __launch_bounds__(PART ? kBaseThreads + kUnpackThreads : kBaseThreads, 1)
 contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                         const ContractionArgs p) {
@@ -164,7 +246,7 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 const long long t0 = clock64();                // let copies in flight land before shared memory is released
                 while (clock64() - t0 < (1ll << 22)) { }
             }
-        } else if (PART && lane == 1) {
+        } else if (PART && !DIRECT && lane == 1) {
             // ---- packed-tile producer: runs ahead of the A loads by up to the depth of its own ring, which
             //      is what hides the latency of fetching the weights
             uint32_t pit = 0;
@@ -308,6 +390,20 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 for (int i = 0; i < SCALES_PER_LANE; ++i) { sc_w[lane + 32 * i] = sc_n[i]; bs_w[lane + 32 * i] = bs_n[i]; }
                 staged_nt = next_nt;
             }
+        }
+    } else if (PART && DIRECT) {
+        // ------------------------------------------------------------------ unpackers reading global memory (h <= 4)
+        PairUnpackCtx cx;
+        cx.sB = sB; cx.full = full; cx.empty = empty; cx.signal_sink = signal_sink; cx.abort_flag = abort_flag;
+        cx.rank = rank; cx.pair = pair; cx.num_pairs = num_pairs; cx.num_tiles = num_tiles;
+        cx.group = (warp - kFirstUnpackWarp) / kUnpackGroupWarps;
+        cx.utid = (threadIdx.x - kBaseThreads) % kUnpackGroupThreads;
+        cx.lane = lane;
+        switch (p.h_bits) {
+            case 1: pair_unpack_direct<MODE, 1>(p, cx); break;
+            case 2: pair_unpack_direct<MODE, 2>(p, cx); break;
+            case 3: pair_unpack_direct<MODE, 3>(p, cx); break;
+            default: pair_unpack_direct<MODE, 4>(p, cx); break;
         }
     } else if (PART) {
         // ------------------------------------------------------------------ unpackers (both CTAs, own half of B)

@@ -89,14 +89,14 @@ int launch_mode(int mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const 
 }
 
 // CTA-pair kernel: a cluster of two CTAs per 256 x 256 tile
-template <bool PART, int MODE>
+template <bool PART, int MODE, bool DIRECT = false>
 int launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const ContractionArgs& a, cudaStream_t stream) {
     const int smem = pair_smem_bytes(PART, a.h_bits, a.packed_stages);
     static int configured[64] = {0};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return NQ_ERR_CUDA;
     if (smem > configured[dev]) {
-        if (cudaFuncSetAttribute(contraction_pair_kernel<PART, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(contraction_pair_kernel<PART, MODE, DIRECT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  smem) != cudaSuccess)
             return NQ_ERR_CUDA;
         configured[dev] = smem;
@@ -116,18 +116,25 @@ int launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const Contractio
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, contraction_pair_kernel<PART, MODE>, tmA, tmB, a) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, contraction_pair_kernel<PART, MODE, DIRECT>, tmA, tmB, a) != cudaSuccess) {
         (void)cudaGetLastError();
         return NQ_ERR_CUDA;
     }
     return NQ_OK;
 }
 
-template <bool PART>
+template <bool PART, bool DIRECT = false>
 int launch_pair_mode(int mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const ContractionArgs& a, cudaStream_t s) {
-    if (mode == kModeConv128) return launch_pair<PART, kModeConv128>(tmA, tmB, a, s);
-    if (mode == kModeConv64) return launch_pair<PART, kModeConv64>(tmA, tmB, a, s);
-    return launch_pair<PART, kModeGemm>(tmA, tmB, a, s);
+    if (mode == kModeConv128) return launch_pair<PART, kModeConv128, DIRECT>(tmA, tmB, a, s);
+    if (mode == kModeConv64) return launch_pair<PART, kModeConv64, DIRECT>(tmA, tmB, a, s);
+    return launch_pair<PART, kModeGemm, DIRECT>(tmA, tmB, a, s);
+}
+
+// NQ_PACKED_RING=1 in the environment keeps every part-bit pair launch on the TMA-fed ring of packed tiles
+// (for comparisons and tests); otherwise h <= 4 reads the packed matrix directly (nq_contraction_pair.cuh).
+bool direct_fetch_enabled() {
+    const char* e = getenv("NQ_PACKED_RING");
+    return !(e && e[0] == '1');
 }
 
 // NQ_SINGLE_CTA=1 in the environment keeps every contraction on the one-CTA-per-tile kernel (for comparisons)
@@ -187,6 +194,7 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
     a.status = status_word();
     if (!a.status) return NQ_ERR_CUDA;
     CUtensorMap tmB;
+    bool direct = false;
     if (part) {
         const int l = n_bits - h_bits;
         a.pow2_l = (float)(1 << l);
@@ -196,14 +204,17 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
         // as deep a ring of packed tiles as shared memory allows: it is what hides the load latency of B
         // (pair kernel: a multiple of its unpack group count, see nq_contraction_pair.cuh)
         a.packed_stages = 0;
+        direct = pair && h_bits <= 4 && direct_fetch_enabled();
         const int step = pair ? kUnpackGroups : 1;
-        for (int d = kMaxPackedStages; d >= step; d -= step)
+        for (int d = direct ? 0 : kMaxPackedStages; d >= step; d -= step)
             if ((pair ? pair_smem_bytes(true, h_bits, d) : contraction_smem_bytes(bn, true, h_bits, d)) <= kSmemLimit) {
                 a.packed_stages = d;
                 break;
             }
-        if (a.packed_stages == 0) return NQ_ERR_UNSUPPORTED;
+        if (a.packed_stages == 0 && !direct) return NQ_ERR_UNSUPPORTED;
         const uint64_t row_bytes = (uint64_t)((K + 127) / 128) * 16 * h_bits;
+        a.packed_b = static_cast<const uint8_t*>(Bmat);      // read directly by the DIRECT pair kernel
+        a.packed_pitch = (long long)row_bytes;
         int st = encode_tensor_map_2d(&tmB, Bmat, row_bytes, (uint64_t)N, row_bytes, 16 * h_bits, b_box_rows, 0);
         if (st != NQ_OK) return st;
     } else {
@@ -213,6 +224,7 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
                      : encode_tensor_map_2d(&tmB, Bmat, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, kBK, b_box_rows, 128);
         if (st != NQ_OK) return st;
     }
+    if (pair && direct) return launch_pair_mode<true, true>(mode, tmA, tmB, a, stream);
     if (pair) return part ? launch_pair_mode<true>(mode, tmA, tmB, a, stream) : launch_pair_mode<false>(mode, tmA, tmB, a, stream);
     if (part) {
         if (bn == 256) return launch_mode<256, true>(mode, tmA, tmB, a, stream);

@@ -60,17 +60,18 @@ def test_config3_whole_model_page_out_and_page_in_in_one_call():
         assert np.array_equal(host(tensors[i]["packed_low"]), oracle.pack_sliced(wlo, n - h + 1))
 
 
-@pytest.mark.parametrize("name", ["l1b0c2", "l1b0c3", "l3b1c1", "l4b0c2"])
-def test_config3_convolution_layers_at_batch_128_sampled_pixels(name):
+@pytest.mark.parametrize("name,h", [("l1b0c2", 6), ("l1b0c3", 6), ("l3b1c1", 6), ("l4b0c2", 6),
+                                    ("l3b1c1", 4), ("l4b0c2", 4), ("l1b0c3", 3)])
+def test_config3_convolution_layers_at_batch_128_sampled_pixels(name, h):
     L = next(l for l in wl.resnet101_layers() if l.name == name)
     batch = 128
     d = wl.conv_layer_inputs(3, 7, L, batch)
     X, W, mask, ws, sa = d["X"], d["W"], d["mask"], d["w_scale"], d["act_scale"]
-    wh, _ = oracle.decompose(W, mask, 8, 6, True)
+    wh, _ = oracle.decompose(W, mask, 8, h, True)
     ldw = -(-L.K // 16) * 16
     w_mat = dev(wl.oihw_to_ohwi_matrix(W, ldw))[:, :L.K]
     m_mat = dev(wl.oihw_to_ohwi_matrix(mask, ldw))[:, :L.K]
-    hi, _ = nq.nq_decompose(w_mat, m_mat, 8, 6, True)
+    hi, _ = nq.nq_decompose(w_mat, m_mat, 8, h, True)
     desc = nq.nq_conv_desc(batch, L.Cin, L.H, L.W, L.Cout, L.R, L.S, L.stride, L.pad, 1)
     rng = wl.rng_for(3, 99)
     Ho, Wo = L.Ho, L.Wo
@@ -80,12 +81,12 @@ def test_config3_convolution_layers_at_batch_128_sampled_pixels(name):
     idx = torch.from_numpy(pix).cuda()
     x_dev, wsd = dev(X), dev(ws)
     for part in (False, True):
-        acc, y, _ = nq.nq_conv_implicit_gemm(x_dev, hi if part else w_mat, desc, wsd, sa, part_bit=part, n_bits=8, h_bits=6,
+        acc, y, _ = nq.nq_conv_implicit_gemm(x_dev, hi if part else w_mat, desc, wsd, sa, part_bit=part, n_bits=8, h_bits=h,
                                              want_acc=True, y_dtype=torch.bfloat16)
         nq.nq_device_status()
         ref = oracle.conv_acc_pixels(X, wh if part else W, L.stride, L.pad, pix)
         assert np.array_equal(host(acc[idx[:, 0], idx[:, 1], idx[:, 2]]), ref)
-        y_ref = oracle.dequant(ref, ws, sa, 2 if part else 0)
+        y_ref = oracle.dequant(ref, ws, sa, 8 - h if part else 0)
         got = host(y[idx[:, 0], idx[:, 1], idx[:, 2]].view(torch.int16)).view(np.uint16)
         assert np.array_equal(got, oracle.f32_to_bf16_bits(y_ref))
 

@@ -129,6 +129,25 @@ def test_full_equals_shifted_part_plus_low_contribution():
     assert torch.equal(full.long(), (part.long() << 3) + low.long())
 
 
+@pytest.mark.parametrize("h", [1, 2, 3, 4])
+def test_wide_ragged_gemm_narrow_fields(h, monkeypatch):
+    """Large enough for the CTA-pair kernel, whose unpack warps read fields of at most 4 bits straight from the
+    packed matrix: ragged in M, N and K, checked against the oracle, and bit for bit against the same launch
+    fed through the shared-memory ring of packed tiles."""
+    M, N, K = 3500, 1100, 1100
+    d = wl.gemm_inputs(89, h, M, N, K)
+    wh, _ = oracle.decompose(d["W"], d["mask"], 8, h, True)
+    hi, _ = nq.nq_decompose(dev_padded(d["W"]), dev_padded(d["mask"]), 8, h, True)
+    Xd, wsd = dev_padded(d["X"]), dev(d["w_scale"])
+    acc, y = nq.nq_gemm_part(Xd, hi, N, 8, h, wsd, d["act_scale"], want_acc=True)
+    nq.nq_device_status()
+    check_outputs(acc, y, oracle.gemm_acc(d["X"], wh), d["w_scale"], d["act_scale"], 8 - h)
+    monkeypatch.setenv("NQ_PACKED_RING", "1")
+    acc2, y2 = nq.nq_gemm_part(Xd, hi, N, 8, h, wsd, d["act_scale"], want_acc=True)
+    nq.nq_device_status()
+    assert torch.equal(acc, acc2) and torch.equal(y, y2)
+
+
 @pytest.mark.parametrize("size,h", [(4096, 6), (4096, 4)])
 def test_large_square_gemm_sampled_rows_and_checksums(size, h):
     """Config-4 shape in the launch configuration the benchmark times: sampled rows bit-exact
