@@ -11,6 +11,11 @@ namespace sm100 {
 
 // A wait that has made no progress for this many SM cycles (about a second) gives up.
 constexpr long long kWaitLimitCycles = 1ll << 31;
+// How long one probe of a barrier may sleep before it reports "not yet" (nanoseconds).  Without a limit a
+// probe sleeps for a period the hardware chooses, and an arrival that comes from the OTHER CTA of a pair (a
+// tcgen05.commit multicast, a remote store) does not cut that sleep short: measured, the partner CTA saw its
+// ring slots freed about 0.8 us late, two stages at a time.
+constexpr uint32_t kTryWaitNs = 40;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -43,10 +48,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred P;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, P;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(kTryWaitNs)
         : "memory");
     return ok != 0;
 }
@@ -209,10 +214,10 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred P;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 P, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 P, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, P;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(kTryWaitNs)
         : "memory");
     return ok != 0;
 }
