@@ -156,6 +156,26 @@ def _run_conv(nq, cs, part):
                                  workspace=cs["work"], y_out=cs["y"])
 
 
+# --------------------------------------------------------------------------- multi-rank arithmetic
+def max_over_ranks(values, world, device=None):
+    """Element-wise maximum over the ranks of a list of per-rank figures (timings): one all-reduce, no data-path
+    collective.  At world 1 the values come back unchanged.  Works on any initialised backend (nccl on GPUs,
+    gloo in the CPU tests)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
+
+
+def whole_job_tops(world, ops_per_gpu_per_step, ms_per_step):
+    """Every rank runs the same per-GPU workload (independent problems, weak scaling): the job's throughput is
+    the ops of all ranks over the slowest rank's time."""
+    return world * ops_per_gpu_per_step / (ms_per_step * 1e-3) / 1e12
+
+
 # --------------------------------------------------------------------------- our arm
 def run_ours(args, rank, world, local_rank):
     import torch
@@ -252,12 +272,9 @@ def run_ours(args, rank, world, local_rank):
     e2e = _run_e2e(nq, torch, sizes, host, state, args, world)
     model_switch = _model_switch(nq, torch, wl, dev) if (rank == 0 and args.model_switch) else None
 
-    if world > 1:
-        t = torch.tensor([total_ms, e2e["ms_per_step"]], device=dev, dtype=torch.float64)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        total_ms, e2e["ms_per_step"] = float(t[0]), float(t[1])
+    total_ms, e2e["ms_per_step"] = max_over_ranks([total_ms, e2e["ms_per_step"]], world, dev)
     ms_per_step = total_ms / args.steps
-    value = world * ops_step / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_tops(world, ops_step, ms_per_step)
     if rank != 0:
         return None
 
@@ -292,7 +309,7 @@ def run_ours(args, rank, world, local_rank):
                                            "between two launches of the same kernel)",
                    "per_gpu_ops_per_step": ops_step},
         "clocks": clocks, "gpu_launches": gpu_launches,
-        "e2e": {"value": round(world * ops_step / (e2e["ms_per_step"] * 1e-3) / 1e12, 3), "unit": "TOPS",
+        "e2e": {"value": round(whole_job_tops(world, ops_step, e2e["ms_per_step"]), 3), "unit": "TOPS",
                 "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                 "ms_per_step": round(e2e["ms_per_step"], 3), "covers": "the GEMM sweep (codec + both GEMM modes)"},
         "roofline": roofline, "rows": rows,
