@@ -9,7 +9,8 @@ One "step" is one pass of the whole path over the large square GEMM sweep (M = N
 followed by the ResNet-18-shaped convolution stack (config 2: 20 convolutions + classifier, batch 32, NCHW
 int8 activations, implicit GEMM, both modes).  After the timed steps the whole-model page-out / page-in of a
 ResNet-101-shaped and a ViT-B-shaped model (one batched launch each, cold L2) is timed separately and
-reported under rows.model_switch.
+reported under rows.model_switch, and configs 3 and 5 run layer by layer through both modes (the ResNet-101-shaped
+stack at batch 128, the ViT-B/16 linears at 256 x 197 tokens): rows.resnet101_stack_int8_6, rows.vit_b16_linears_int8_4.
 `value` is the integer-op throughput of the whole step (2*M*N*K per contraction; the codec kernels
 add time but no ops) in TOPS, summed over ranks.  Per-row numbers (TOPS per mode, GB/s per codec
 kernel) are reported under "rows".
@@ -271,6 +272,7 @@ def run_ours(args, rank, world, local_rank):
 
     e2e = _run_e2e(nq, torch, sizes, host, state, args, world)
     model_switch = _model_switch(nq, torch, wl, dev) if (rank == 0 and args.model_switch) else None
+    model_rows = _model_rows(nq, torch, wl, dev, args.model_batch) if (rank == 0 and args.model_rows and have_conv) else None
 
     total_ms, e2e["ms_per_step"] = max_over_ranks([total_ms, e2e["ms_per_step"]], world, dev)
     ms_per_step = total_ms / args.steps
@@ -316,6 +318,8 @@ def run_ours(args, rank, world, local_rank):
     }
     if model_switch is not None:
         line["rows"]["model_switch"] = model_switch
+    if model_rows is not None:
+        line["rows"].update(model_rows)
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(sizes, host, args.cpu_rows)
     return line
@@ -404,6 +408,106 @@ def _model_switch(nq, torch, wl, dev):
         res["tensors"] = len(shapes)
         res["algorithmic_mb"] = round(nbytes / 1e6, 1)
         out[name] = res
+    return out
+
+
+def _device_conv_weights(torch, L, dev, gen):
+    """[Cout, K] int8 weights of a layer, Gaussian fit then per-channel INT8 quantisation (Eq. 1), generated on the
+    device for the timing-only rows (the parity tests use the seeded host generators)."""
+    ldw = -(-L.K // 16) * 16
+    w = torch.randn((L.Cout, ldw), device=dev, generator=gen) * (2.0 / L.K) ** 0.5
+    s = w[:, :L.K].abs().amax(dim=1).clamp_min(1e-12) / 127.0
+    q = torch.clamp(torch.round(w / s[:, None]), -128, 127).to(torch.int8)
+    q[:, L.K:] = 0
+    return q[:, :L.K], s.float()
+
+
+def _model_rows(nq, torch, wl, dev, conv_batch):
+    """Configs 3 and 5 through both modes, layer by layer on seeded device-side inputs of the stated shapes and
+    distributions: the ResNet-101-shaped stack (104 convolutions + classifier, batch `conv_batch`, NCHW int8
+    activations ~ U{0..127}, INT8 nesting INT6, bf16 out) and the ViT-B/16 linears (M = 256 * 197 tokens, INT8
+    nesting INT4).  Each layer is timed with its own pair of CUDA events, median of 3 passes; inputs of one pass
+    exceed L2, so nothing is flushed."""
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(wl.BASE_SEED + 3000)
+    out = {}
+    # ---- config 3
+    layers = wl.resnet101_layers()
+    xs, prepared = {}, []
+    y_elems = max(conv_batch * L.Ho * L.Wo * L.Cout for L in layers)
+    ybuf = torch.empty(y_elems, dtype=torch.bfloat16, device=dev)
+    work_bytes = 0
+    for L in layers:
+        key = (L.Cin, L.H, L.W)
+        if key not in xs:
+            xs[key] = torch.randint(0, 128, (conv_batch, L.Cin, L.H, L.W), dtype=torch.int8, device=dev, generator=gen)
+        desc = nq.nq_conv_desc(conv_batch, L.Cin, L.H, L.W, L.Cout, L.R, L.S, L.stride, L.pad, 1)
+        w, ws = _device_conv_weights(torch, L, dev, gen)
+        m = torch.randint(0, 2, (L.Cout, w.stride(0)), dtype=torch.uint8, device=dev, generator=gen)[:, :L.K]
+        hi, _ = nq.nq_decompose(w, m, N_BITS, CONV_H, True)
+        work_bytes = max(work_bytes, nq.nq_conv_workspace_bytes(desc))
+        prepared.append({"desc": desc, "w": w, "hi": hi, "ws": ws, "x": xs[key], "act": 0.02,
+                         "y": ybuf[:conv_batch * L.Ho * L.Wo * L.Cout].view(conv_batch, L.Ho, L.Wo, L.Cout)})
+    work = torch.empty(work_bytes + 2048, dtype=torch.uint8, device=dev)
+    for cs in prepared:
+        cs["work"] = work
+    ops = sum(2.0 * float(np.prod(L.gemm_view(conv_batch))) for L in layers)
+    res = {}
+    for part in (False, True):
+        per_layer = []
+        for rep in range(4):
+            evs = []
+            for cs in prepared:
+                a = torch.cuda.Event(enable_timing=True)
+                b = torch.cuda.Event(enable_timing=True)
+                a.record()
+                _run_conv(nq, cs, part)
+                b.record()
+                evs.append((a, b))
+            torch.cuda.synchronize()
+            if rep:
+                per_layer.append([a.elapsed_time(b) for a, b in evs])
+        ms = float(np.sum(np.median(np.array(per_layer), axis=0)))
+        res["part_bit" if part else "full_bit"] = {"ms": round(ms, 3), "tops": round(ops / (ms * 1e-3) / 1e12, 1)}
+    res.update({"layers": len(layers), "batch": conv_batch, "weights": sum(L.weights for L in layers),
+                "tera_ops_per_pass": round(ops / 1e12, 3)})
+    out["resnet101_stack_int8_6"] = res
+    nq.nq_device_status()
+    del prepared, xs, ybuf, work
+    torch.cuda.empty_cache()
+    # ---- config 5
+    M = 256 * wl.VIT_TOKENS
+    res = {}
+    for _, k, n in wl.vit_b16_linears(1):
+        x = torch.clamp(torch.round(torch.randn((M, k), device=dev, generator=gen) * 32.0), -128, 127).to(torch.int8)
+        wf = torch.randn((n, k), device=dev, generator=gen) * 0.02
+        hit = torch.rand((n, k), device=dev, generator=gen) < 1e-3
+        sign = torch.where(torch.rand((n, k), device=dev, generator=gen) < 0.5, -1.0, 1.0)
+        wf = torch.where(hit, sign * 0.12, wf)
+        sc = wf.abs().amax(dim=1) / 127.0
+        w = torch.clamp(torch.round(wf / sc[:, None]), -128, 127).to(torch.int8)
+        m = torch.randint(0, 2, w.shape, dtype=torch.uint8, device=dev, generator=gen)
+        hi, _ = nq.nq_decompose(w, m, N_BITS, 4, True)
+        y = torch.empty((M, n), dtype=torch.bfloat16, device=dev)
+        row = {}
+        for name, fn in (("full_bit", lambda: nq.nq_gemm_full(x, w, sc, ACT_SCALE, y_out=y)),
+                         ("part_bit", lambda: nq.nq_gemm_part(x, hi, n, N_BITS, 4, sc, ACT_SCALE, y_out=y))):
+            ts = []
+            for rep in range(5):
+                a = torch.cuda.Event(enable_timing=True)
+                b = torch.cuda.Event(enable_timing=True)
+                a.record()
+                fn()
+                b.record()
+                torch.cuda.synchronize()
+                if rep:
+                    ts.append(a.elapsed_time(b))
+            ms = float(np.median(ts))
+            row[name] = {"ms": round(ms, 4), "tops": round(2.0 * M * n * k / (ms * 1e-3) / 1e12, 1)}
+        res[f"K{k}_N{n}"] = row
+    res["M"] = M
+    out["vit_b16_linears_int8_4"] = res
+    nq.nq_device_status()
     return out
 
 
@@ -517,6 +621,9 @@ def main():
     ap.add_argument("--no-conv", dest="conv", action="store_false")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-model-switch", dest="model_switch", action="store_false")
+    ap.add_argument("--no-model-rows", dest="model_rows", action="store_false",
+                    help="skip the ResNet-101-shaped stack and the ViT-B linears (timed after the steps)")
+    ap.add_argument("--model-batch", type=int, default=128)
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
