@@ -69,6 +69,7 @@ struct ContractionArgs {
     void* y;
     long long ldy;
     int y_is_bf16;
+    int y_tma, acc_tma;  // the output is written with tile stores through tmY / tmAcc (aligned base and pitch)
     unsigned int* status;
 };
 
@@ -329,13 +330,41 @@ __device__ __forceinline__ void store_rows64(uint8_t* stage, int lane, const uin
     __syncwarp();
 }
 
+// Where the 32 rows of an epilogue warp sit in the output, as tile-store coordinates (dimensions 1..3 of the
+// output map; dimension 0 is the byte offset of the columns).
+struct OutCoords {
+    int c1, c2, c3;
+};
+// The same 32 x 64-byte block handed to the TMA unit instead: the lanes lay their rows down in the 64-byte
+// swizzle (no bank conflicts), one lane issues a tile store, and nobody reads the block back or issues a global
+// store -- the load/store unit was the busiest unit of output-bound problems, and most of its shared-memory
+// traffic was that read-back.  Rows and columns outside the output are clipped by the store.
+// The buffer is reused once the previous store from it has finished reading.
+__device__ __forceinline__ void store_rows64_tma(uint8_t* stage, int lane, const uint4 (&q)[4], const CUtensorMap* map,
+                                                 int x_byte, const OutCoords& oc) {
+    using namespace sm100;
+    if (lane == 0) bulk_wait_read_all();
+    __syncwarp();
+    uint8_t* mine = stage + lane * 64;
+    const int sw = (lane >> 1) & 3;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4*>(mine + ((j ^ sw) << 4)) = q[j];
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+        tma_store_4d(map, smem_u32(stage), x_byte, oc.c1, oc.c2, oc.c3);
+        bulk_commit_group();
+    }
+}
+
 // The epilogue of one warp for 32 consecutive columns: same arithmetic as store_chunk, coalesced stores.
 __device__ __forceinline__ void store_chunk_warp(const ContractionArgs& p, int row, bool row_ok, int col0,
                                                  const uint32_t (&r)[32], const float* sc, const float* bs,
-                                                 bool vec_acc, bool vec_f32, bool vec_bf16, uint8_t* stage, int lane) {
+                                                 bool vec_acc, bool vec_f32, bool vec_bf16, uint8_t* stage, int lane,
+                                                 const CUtensorMap* tmY, const CUtensorMap* tmAcc, const OutCoords& oc) {
     const bool full_chunk = col0 + 32 <= p.N;
-    const bool acc_fast = p.acc_out == nullptr || (full_chunk && vec_acc);
-    const bool y_fast = p.y == nullptr || (full_chunk && (p.y_is_bf16 ? vec_bf16 : vec_f32));
+    const bool acc_fast = p.acc_out == nullptr || p.acc_tma || (full_chunk && vec_acc);
+    const bool y_fast = p.y == nullptr || p.y_tma || (full_chunk && (p.y_is_bf16 ? vec_bf16 : vec_f32));
     if (!acc_fast || !y_fast) {                        // ragged or unaligned: the plain per-row path
         if (row_ok) store_chunk(p, row, col0, r, sc, bs, vec_acc, vec_f32, vec_bf16);
         return;
@@ -348,8 +377,9 @@ __device__ __forceinline__ void store_chunk_warp(const ContractionArgs& p, int r
             for (int j = 0; j < 4; ++j)
                 q[j] = make_uint4((uint32_t)((int)r[half * 16 + 4 * j] >> p.acc_shift), (uint32_t)((int)r[half * 16 + 4 * j + 1] >> p.acc_shift),
                                   (uint32_t)((int)r[half * 16 + 4 * j + 2] >> p.acc_shift), (uint32_t)((int)r[half * 16 + 4 * j + 3] >> p.acc_shift));
-            store_rows64(stage, lane, q, row, row_ok, reinterpret_cast<uint8_t*>(p.acc_out), p.ld_acc * 4,
-                         (long long)(col0 + half * 16) * 4);
+            if (p.acc_tma) store_rows64_tma(stage, lane, q, tmAcc, (col0 + half * 16) * 4, oc);
+            else store_rows64(stage, lane, q, row, row_ok, reinterpret_cast<uint8_t*>(p.acc_out), p.ld_acc * 4,
+                              (long long)(col0 + half * 16) * 4);
         }
     }
     if (p.y) {
@@ -381,8 +411,9 @@ __device__ __forceinline__ void store_chunk_warp(const ContractionArgs& p, int r
                 for (int j = 0; j < 4; ++j)
                     q[j] = make_uint4(__float_as_uint(v[half * 16 + 4 * j]), __float_as_uint(v[half * 16 + 4 * j + 1]),
                                       __float_as_uint(v[half * 16 + 4 * j + 2]), __float_as_uint(v[half * 16 + 4 * j + 3]));
-                store_rows64(stage, lane, q, row, row_ok, reinterpret_cast<uint8_t*>(p.y), p.ldy * 4,
-                             (long long)(col0 + half * 16) * 4);
+                if (p.y_tma) store_rows64_tma(stage, lane, q, tmY, (col0 + half * 16) * 4, oc);
+                else store_rows64(stage, lane, q, row, row_ok, reinterpret_cast<uint8_t*>(p.y), p.ldy * 4,
+                                  (long long)(col0 + half * 16) * 4);
             }
         } else {
 #pragma unroll
@@ -394,9 +425,25 @@ __device__ __forceinline__ void store_chunk_warp(const ContractionArgs& p, int r
                 q[j] = make_uint4(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b),
                                   *reinterpret_cast<uint32_t*>(&c2), *reinterpret_cast<uint32_t*>(&d));
             }
-            store_rows64(stage, lane, q, row, row_ok, reinterpret_cast<uint8_t*>(p.y), p.ldy * 2, (long long)col0 * 2);
+            if (p.y_tma) store_rows64_tma(stage, lane, q, tmY, col0 * 2, oc);
+            else store_rows64(stage, lane, q, row, row_ok, reinterpret_cast<uint8_t*>(p.y), p.ldy * 2, (long long)col0 * 2);
         }
     }
+}
+
+// Tile-store coordinates of the 32 rows that start at tile row ml0 (a multiple of 32) of M-tile mt.
+template <int MODE>
+__device__ __forceinline__ OutCoords out_coords(const ContractionArgs& p, int mt, int ml0) {
+    OutCoords oc;
+    if (MODE == kModeGemm) {
+        oc.c1 = mt * kBM + ml0; oc.c2 = 0; oc.c3 = 0;
+    } else {
+        const TileOrigin o = conv_tile_origin(p.g, mt);
+        oc.c1 = o.q0 + (ml0 & ((1 << p.g.tw_log2) - 1));
+        oc.c2 = o.p0 + ((ml0 >> p.g.tw_log2) & ((1 << p.g.th_log2) - 1));
+        oc.c3 = o.b0 + (ml0 >> (p.g.tw_log2 + p.g.th_log2));
+    }
+    return oc;
 }
 
 // Per-channel output factors of 32 * PER_LANE consecutive columns starting at col_base, lane-strided:
@@ -419,6 +466,7 @@ __device__ __forceinline__ void fetch_scales(const ContractionArgs& p, int col_b
 template <int BN, bool PART, int MODE>
 __global__ void __launch_bounds__(PART ? kBaseThreads + kUnpackThreads : kBaseThreads, 1)
 contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                   const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmAcc,
                    const ContractionArgs p) {
     using namespace sm100;
     constexpr int STAGES = stages_for(BN, PART);
@@ -468,6 +516,8 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         fence_barrier_init();
         prefetch_tensormap(&tmA);
         prefetch_tensormap(&tmB);
+        if (p.y_tma) prefetch_tensormap(&tmY);
+        if (p.acc_tma) prefetch_tensormap(&tmAcc);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
@@ -640,6 +690,7 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 row_ok = qq < p.g.Wo && pp < p.g.Ho && bb < p.g.B;
                 row = ((long long)bb * p.g.Ho + pp) * p.g.Wo + qq;
             }
+            const OutCoords oc = out_coords<MODE>(p, mt, quarter * 32);
             constexpr int CHUNKS = BN / 64;                // 32-column chunks per warp (half of the tile)
 #pragma unroll 1
             for (int cc = 0; cc < CHUNKS; ++cc) {
@@ -655,7 +706,7 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 const int col0 = n0 + c * 32;
                 if (col0 >= p.N) continue;
                 store_chunk_warp(p, (int)row, row_ok, col0, r, sc_w + cc * 32, bs_w + cc * 32, vec_acc, vec_f32, vec_bf16,
-                                 sStage + (warp - 2) * kEpiStageBytes, lane);
+                                 sStage + (warp - 2) * kEpiStageBytes, lane, &tmY, &tmAcc, oc);
             }
             if (next_nt >= 0 && next_nt != nt) {
                 __syncwarp();
@@ -664,6 +715,7 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 staged_nt = next_nt;
             }
         }
+        if (lane == 0) bulk_wait_all();                    // this lane's tile stores are done before the block leaves
     } else if (PART) {
         // ------------------------------------------------------------------ unpackers (warps 6-13)
         const int utid = threadIdx.x - kBaseThreads;

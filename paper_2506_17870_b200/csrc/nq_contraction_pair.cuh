@@ -136,6 +136,7 @@ __device__ __forceinline__ void pair_unpack_direct(const ContractionArgs& p, con
 template <bool PART, int MODE, bool DIRECT = false>
 __global__ void __launch_bounds__(PART ? kBaseThreads + kUnpackThreads : kBaseThreads, 1)
 contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                        const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmAcc,
                         const ContractionArgs p) {
     using namespace sm100;
     constexpr int BN = kPairBN;
@@ -189,6 +190,8 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         fence_barrier_init();
         prefetch_tensormap(&tmA);
         prefetch_tensormap(&tmB);
+        if (p.y_tma) prefetch_tensormap(&tmY);
+        if (p.acc_tma) prefetch_tensormap(&tmAcc);
     }
     if (warp == 1) {
         tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS);
@@ -364,6 +367,7 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 row_ok = qq < p.g.Wo && pp < p.g.Ho && bb < p.g.B;
                 row = ((long long)bb * p.g.Ho + pp) * p.g.Wo + qq;
             }
+            const OutCoords oc = out_coords<MODE>(p, mt, quarter * 32);
             constexpr int CHUNKS = BN / 64;                // 32-column chunks per warp (half of the tile)
 #pragma unroll 1
             for (int cc = 0; cc < CHUNKS; ++cc) {
@@ -382,7 +386,7 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 const int col0 = n0 + c * 32;
                 if (col0 >= p.N) continue;
                 store_chunk_warp(p, (int)row, row_ok, col0, r, sc_w + cc * 32, bs_w + cc * 32, vec_acc, vec_f32, vec_bf16,
-                                 sStage + (warp - 2) * kEpiStageBytes, lane);
+                                 sStage + (warp - 2) * kEpiStageBytes, lane, &tmY, &tmAcc, oc);
             }
             if (next_nt >= 0 && next_nt != nt) {
                 __syncwarp();
@@ -391,6 +395,7 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 staged_nt = next_nt;
             }
         }
+        if (lane == 0) bulk_wait_all();                    // this lane's tile stores are done before the block leaves
     } else if (PART && DIRECT) {
         // ------------------------------------------------------------------ unpackers reading global memory (h <= 4)
         PairUnpackCtx cx;

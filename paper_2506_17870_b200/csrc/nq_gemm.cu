@@ -61,10 +61,30 @@ int encode_tensor_map_nhwc(CUtensorMap* map, const void* base, uint64_t C, uint6
     return r == CUDA_SUCCESS ? NQ_OK : NQ_ERR_CUDA;
 }
 
+int encode_tensor_map_out(CUtensorMap* map, const void* base, uint64_t row_bytes, uint64_t pitch_bytes, uint64_t d1,
+                          uint64_t d2, uint64_t d3, uint32_t b1, uint32_t b2, uint32_t b3) {
+    EncodeFn fn = encode_fn();
+    if (!fn) return NQ_ERR_CUDA;
+    cuuint64_t dims[4] = {row_bytes, d1, d2, d3};
+    cuuint64_t strides[3] = {pitch_bytes, pitch_bytes * d1, pitch_bytes * d1 * d2};
+    cuuint32_t box[4] = {64, b1, b2, b3};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? NQ_OK : NQ_ERR_CUDA;
+}
+
 namespace {
 
+// The two output maps of a launch (Y and the int32 accumulators); a map that is not used is a copy of tmA, so
+// that the kernel parameter is always a valid descriptor.
+struct OutMaps {
+    CUtensorMap y, acc;
+};
+
 template <int BN, bool PART, int MODE>
-int launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const ContractionArgs& a, cudaStream_t stream) {
+int launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const OutMaps& om, const ContractionArgs& a, cudaStream_t stream) {
     const int smem = contraction_smem_bytes(BN, PART, a.h_bits, a.packed_stages);
     static int configured[64] = {0};       // largest opt-in done so far, per device, for this instantiation
     int dev = 0;
@@ -77,20 +97,22 @@ int launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const ContractionArgs
     }
     const int tiles = a.m_tiles * a.n_tiles;
     const int grid = tiles < sm_count() ? tiles : sm_count();
-    contraction_kernel<BN, PART, MODE><<<grid, PART ? kBaseThreads + kUnpackThreads : kBaseThreads, smem, stream>>>(tmA, tmB, a);
+    contraction_kernel<BN, PART, MODE><<<grid, PART ? kBaseThreads + kUnpackThreads : kBaseThreads, smem, stream>>>(tmA, tmB, om.y, om.acc, a);
     return cudaGetLastError() == cudaSuccess ? NQ_OK : NQ_ERR_CUDA;
 }
 
 template <int BN, bool PART>
-int launch_mode(int mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const ContractionArgs& a, cudaStream_t s) {
-    if (mode == kModeConv128) return launch<BN, PART, kModeConv128>(tmA, tmB, a, s);
-    if (mode == kModeConv64) return launch<BN, PART, kModeConv64>(tmA, tmB, a, s);
-    return launch<BN, PART, kModeGemm>(tmA, tmB, a, s);
+int launch_mode(int mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const OutMaps& om, const ContractionArgs& a,
+                cudaStream_t s) {
+    if (mode == kModeConv128) return launch<BN, PART, kModeConv128>(tmA, tmB, om, a, s);
+    if (mode == kModeConv64) return launch<BN, PART, kModeConv64>(tmA, tmB, om, a, s);
+    return launch<BN, PART, kModeGemm>(tmA, tmB, om, a, s);
 }
 
 // CTA-pair kernel: a cluster of two CTAs per 256 x 256 tile
 template <bool PART, int MODE, bool DIRECT = false>
-int launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const ContractionArgs& a, cudaStream_t stream) {
+int launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const OutMaps& om, const ContractionArgs& a,
+                cudaStream_t stream) {
     const int smem = pair_smem_bytes(PART, a.h_bits, a.packed_stages);
     static int configured[64] = {0};
     int dev = 0;
@@ -116,7 +138,7 @@ int launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const Contractio
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, contraction_pair_kernel<PART, MODE, DIRECT>, tmA, tmB, a) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, contraction_pair_kernel<PART, MODE, DIRECT>, tmA, tmB, om.y, om.acc, a) != cudaSuccess) {
         (void)cudaGetLastError();
         return NQ_ERR_CUDA;
     }
@@ -124,10 +146,32 @@ int launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const Contractio
 }
 
 template <bool PART, bool DIRECT = false>
-int launch_pair_mode(int mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const ContractionArgs& a, cudaStream_t s) {
-    if (mode == kModeConv128) return launch_pair<PART, kModeConv128, DIRECT>(tmA, tmB, a, s);
-    if (mode == kModeConv64) return launch_pair<PART, kModeConv64, DIRECT>(tmA, tmB, a, s);
-    return launch_pair<PART, kModeGemm, DIRECT>(tmA, tmB, a, s);
+int launch_pair_mode(int mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const OutMaps& om, const ContractionArgs& a,
+                     cudaStream_t s) {
+    if (mode == kModeConv128) return launch_pair<PART, kModeConv128, DIRECT>(tmA, tmB, om, a, s);
+    if (mode == kModeConv64) return launch_pair<PART, kModeConv64, DIRECT>(tmA, tmB, om, a, s);
+    return launch_pair<PART, kModeGemm, DIRECT>(tmA, tmB, om, a, s);
+}
+
+// NQ_PLAIN_STORES=1 in the environment keeps the epilogue on ordinary global stores (for comparisons and tests)
+bool tile_stores_enabled() {
+    const char* e = getenv("NQ_PLAIN_STORES");
+    return !(e && e[0] == '1');
+}
+
+// Tile-store map of one output ([M, N] of esize-byte elements, pitch ld): possible when base and pitch are
+// 16-byte aligned.  Convolution outputs are NHWC, addressed by (pixel column, pixel row, image) in boxes that
+// match the 32 consecutive tile rows of an epilogue warp.
+bool make_out_map(CUtensorMap* map, const void* base, int esize, int64_t M, int64_t N, int64_t ld, const ConvGeom* g) {
+    if (!base || !tile_stores_enabled()) return false;
+    const uint64_t pitch = (uint64_t)ld * esize, row_bytes = (uint64_t)N * esize;
+    if ((reinterpret_cast<uintptr_t>(base) & 15) || (pitch & 15) || pitch >= (1ull << 40)) return false;
+    if (!g) return encode_tensor_map_out(map, base, row_bytes, pitch, (uint64_t)M, 1, 1, 32, 1, 1) == NQ_OK;
+    const uint32_t tw = 1u << g->tw_log2, th = 1u << g->th_log2;
+    const uint32_t bw = tw < 32 ? tw : 32;
+    const uint32_t bh = (32 / bw) < th ? (32 / bw) : th;
+    const uint32_t bb = 32 / (bw * bh);
+    return encode_tensor_map_out(map, base, row_bytes, pitch, (uint64_t)g->Wo, (uint64_t)g->Ho, (uint64_t)g->B, bw, bh, bb) == NQ_OK;
 }
 
 // NQ_PACKED_RING=1 in the environment keeps every part-bit pair launch on the TMA-fed ring of packed tiles
@@ -193,6 +237,10 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
     a.acc_out = acc_out; a.ld_acc = ld_acc; a.y = Y; a.ldy = ldy; a.y_is_bf16 = (y_dtype == NQ_BF16);
     a.status = status_word();
     if (!a.status) return NQ_ERR_CUDA;
+    OutMaps om;
+    om.y = tmA; om.acc = tmA;
+    a.y_tma = make_out_map(&om.y, Y, y_dtype == NQ_BF16 ? 2 : 4, M, N, ldy, geom) ? 1 : 0;
+    a.acc_tma = make_out_map(&om.acc, acc_out, 4, M, N, ld_acc, geom) ? 1 : 0;
     CUtensorMap tmB;
     bool direct = false;
     if (part) {
@@ -224,16 +272,16 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
                      : encode_tensor_map_2d(&tmB, Bmat, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, kBK, b_box_rows, 128);
         if (st != NQ_OK) return st;
     }
-    if (pair && direct) return launch_pair_mode<true, true>(mode, tmA, tmB, a, stream);
-    if (pair) return part ? launch_pair_mode<true>(mode, tmA, tmB, a, stream) : launch_pair_mode<false>(mode, tmA, tmB, a, stream);
+    if (pair && direct) return launch_pair_mode<true, true>(mode, tmA, tmB, om, a, stream);
+    if (pair) return part ? launch_pair_mode<true>(mode, tmA, tmB, om, a, stream) : launch_pair_mode<false>(mode, tmA, tmB, om, a, stream);
     if (part) {
-        if (bn == 256) return launch_mode<256, true>(mode, tmA, tmB, a, stream);
-        if (bn == 128) return launch_mode<128, true>(mode, tmA, tmB, a, stream);
-        return launch_mode<64, true>(mode, tmA, tmB, a, stream);
+        if (bn == 256) return launch_mode<256, true>(mode, tmA, tmB, om, a, stream);
+        if (bn == 128) return launch_mode<128, true>(mode, tmA, tmB, om, a, stream);
+        return launch_mode<64, true>(mode, tmA, tmB, om, a, stream);
     }
-    if (bn == 256) return launch_mode<256, false>(mode, tmA, tmB, a, stream);
-    if (bn == 128) return launch_mode<128, false>(mode, tmA, tmB, a, stream);
-    return launch_mode<64, false>(mode, tmA, tmB, a, stream);
+    if (bn == 256) return launch_mode<256, false>(mode, tmA, tmB, om, a, stream);
+    if (bn == 128) return launch_mode<128, false>(mode, tmA, tmB, om, a, stream);
+    return launch_mode<64, false>(mode, tmA, tmB, om, a, stream);
 }
 
 namespace {

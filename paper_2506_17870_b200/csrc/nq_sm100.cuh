@@ -93,6 +93,25 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n)
         : "memory");
 }
+// 4-D tile store from this CTA's shared memory; elements outside the tensor are not written.  Tracked by the
+// issuing thread's bulk async-group.
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+        ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() {
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// the issuing thread's tile stores have all finished READING shared memory (the buffer may be rewritten)
+__device__ __forceinline__ void bulk_wait_read_all() {
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+// ... and have all completed
+__device__ __forceinline__ void bulk_wait_all() {
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
 // generic-proxy writes to shared memory -> visible to the async proxy (TMA, tcgen05.mma)
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -291,5 +310,9 @@ int encode_tensor_map_2d(CUtensorMap* map, const void* base, uint64_t inner, uin
 // pixels taken every `stride` input pixels.
 int encode_tensor_map_nhwc(CUtensorMap* map, const void* base, uint64_t C, uint64_t W, uint64_t H, uint64_t B,
                            uint32_t box_c, uint32_t tw, uint32_t th, uint32_t tb, uint32_t stride, int swizzle_bytes);
+// Output matrix as a 4-D byte tensor (row bytes, d1, d2, d3) for the epilogue's tile stores: boxes of 64 bytes x
+// b1 x b2 x b3 rows (32 rows in all) in the 64-byte swizzle.  A plain [M, N] matrix is (N * esize, M, 1, 1).
+int encode_tensor_map_out(CUtensorMap* map, const void* base, uint64_t row_bytes, uint64_t pitch_bytes, uint64_t d1,
+                          uint64_t d2, uint64_t d3, uint32_t b1, uint32_t b2, uint32_t b3);
 
 }  // namespace nq
