@@ -85,6 +85,24 @@ def test_other_nestings(h):
     run_layer(C("c128", 128, 8, 8, 64, 3, 3, 1, 1), 4, 20 + h, h=h)
 
 
+@pytest.mark.parametrize("L", [C("c64_wide", 64, 40, 40, 64, 3, 3, 1, 1), C("c128_ragged", 128, 13, 9, 72, 3, 3, 2, 1)],
+                         ids=lambda l: l.name)
+def test_tile_stores_and_plain_stores_agree(L, monkeypatch):
+    """NHWC outputs go out as 4-D tile stores whose boxes follow the pixel rectangle of a tile (pixels outside the
+    image are clipped by the store); the ordinary-store epilogue must give the same bytes."""
+    run_layer(L, 3, 77)
+    d = wl.conv_layer_inputs(71, 78, L, 3)
+    ldw = -(-L.K // 16) * 16
+    w_mat = dev(wl.oihw_to_ohwi_matrix(d["W"], ldw))[:, :L.K]
+    desc = nq.nq_conv_desc(3, L.Cin, L.H, L.W, L.Cout, L.R, L.S, L.stride, L.pad, 1)
+    x, ws = dev(d["X"]), dev(d["w_scale"])
+    acc, y, _ = nq.nq_conv_implicit_gemm(x, w_mat, desc, ws, 0.02, want_acc=True, y_dtype=torch.bfloat16)
+    monkeypatch.setenv("NQ_PLAIN_STORES", "1")
+    acc2, y2, _ = nq.nq_conv_implicit_gemm(x, w_mat, desc, ws, 0.02, want_acc=True, y_dtype=torch.bfloat16)
+    nq.nq_device_status()
+    assert torch.equal(acc, acc2) and torch.equal(y.view(torch.int16), y2.view(torch.int16))
+
+
 def test_pointwise_convolution_equals_the_gemm_entry_point():
     L = C("pw", 128, 6, 6, 96, 1, 1, 1, 0)
     d = wl.conv_layer_inputs(72, 0, L, 5)

@@ -148,6 +148,24 @@ def test_wide_ragged_gemm_narrow_fields(h, monkeypatch):
     assert torch.equal(acc, acc2) and torch.equal(y, y2)
 
 
+@pytest.mark.parametrize("M,N,K,bf16", [(300, 520, 1000, False), (300, 520, 1000, True), (1030, 1100, 640, True),
+                                         (130, 40, 147, False), (2100, 72, 256, True)])
+def test_tile_stores_and_plain_stores_agree(M, N, K, bf16, monkeypatch):
+    """The epilogue writes aligned outputs with TMA tile stores (ragged rows and columns clipped by the store) and
+    everything else with ordinary stores: both against the oracle, and bit for bit against each other."""
+    d = wl.gemm_inputs(90, M + N + K, M, N, K)
+    run_both_modes(d, 8, 6, bf16=bf16)
+    hi, _ = nq.nq_decompose(dev_padded(d["W"]), dev_padded(d["mask"]), 8, 6, True)
+    Xd, wsd = dev_padded(d["X"]), dev(d["w_scale"])
+    ydt = torch.bfloat16 if bf16 else torch.float32
+    acc, y = nq.nq_gemm_part(Xd, hi, N, 8, 6, wsd, d["act_scale"], want_acc=True, y_dtype=ydt)
+    monkeypatch.setenv("NQ_PLAIN_STORES", "1")
+    acc2, y2 = nq.nq_gemm_part(Xd, hi, N, 8, 6, wsd, d["act_scale"], want_acc=True, y_dtype=ydt)
+    nq.nq_device_status()
+    assert torch.equal(acc, acc2) and torch.equal(y.view(torch.int16 if bf16 else torch.int32),
+                                                  y2.view(torch.int16 if bf16 else torch.int32))
+
+
 @pytest.mark.parametrize("size,h", [(4096, 6), (4096, 4)])
 def test_large_square_gemm_sampled_rows_and_checksums(size, h):
     """Config-4 shape in the launch configuration the benchmark times: sampled rows bit-exact
