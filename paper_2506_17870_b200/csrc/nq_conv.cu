@@ -23,38 +23,59 @@ static __device__ __align__(256) unsigned char g_conv_static_scratch[NQ_CONV_STA
 namespace nq {
 namespace {
 
-// [B, C, HW] int8 -> [B, HW, C]; a block moves 64 channels x 64 pixels through shared memory
+// [B, C, HW] int8 -> [B, HW, C]; a block moves 64 channels x 128 pixels.  A thread loads one word (four pixels)
+// of each of eight channels -- a warp's load is 128 contiguous bytes of one channel -- turns them into the eight
+// channel bytes of each of its four pixels with byte permutes in registers (two 4 x 4 byte transposes), and
+// parks those in shared memory, from where whole 16-byte pieces of pixel rows go out.  (Scattering single bytes
+// into shared memory, as a first version did, ran at under a third of the memory bandwidth.)
 __global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(const int8_t* __restrict__ in, int8_t* __restrict__ out,
                                                            int C, int HW) {
-    __shared__ __align__(16) uint8_t tile[64][80];            // [pixel][channel], pitch 80 keeps rows 16-byte aligned
-    const int b = blockIdx.z, c0 = blockIdx.y * 64, p0 = blockIdx.x * 64;
+    __shared__ __align__(16) uint8_t tile[128][80];           // [pixel slot][channel]; pixel p sits in slot (p % 4) * 32 + p / 4
+    const int b = blockIdx.z, c0 = blockIdx.y * 64, p0 = blockIdx.x * 128;
     const int8_t* src = in + ((size_t)b * C + c0) * HW;
     int8_t* dst = out + (size_t)b * HW * C;
     const int t = threadIdx.x;
+    const int pq = t & 31, cg = t >> 5;                       // pixel quad of the block, group of eight channels
     const bool words = ((HW & 3) == 0) && ((reinterpret_cast<uintptr_t>(in) & 3) == 0);
+    const int px = p0 + 4 * pq;
+    uint32_t w[8];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int c = (t >> 4) + 16 * i, x4 = (t & 15) * 4;
-        uint32_t w = 0;
-        if (c0 + c < C) {
-            if (words && p0 + x4 + 3 < HW) {
-                w = *reinterpret_cast<const uint32_t*>(src + (size_t)c * HW + p0 + x4);
+    for (int k = 0; k < 8; ++k) {
+        const int c = cg * 8 + k;
+        uint32_t v = 0;
+        if (c0 + c < C && px < HW) {
+            if (words) {                                       // HW is a multiple of 4, so the whole quad is inside
+                v = __ldg(reinterpret_cast<const uint32_t*>(src + (size_t)c * HW + px));
             } else {
                 for (int j = 0; j < 4; ++j)
-                    if (p0 + x4 + j < HW) w |= (uint32_t)(uint8_t)src[(size_t)c * HW + p0 + x4 + j] << (8 * j);
+                    if (px + j < HW) v |= (uint32_t)(uint8_t)src[(size_t)c * HW + px + j] << (8 * j);
             }
         }
-#pragma unroll
-        for (int j = 0; j < 4; ++j) tile[x4 + j][c] = (uint8_t)(w >> (8 * j));
+        w[k] = v;
     }
+    uint32_t o[4][2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const uint32_t t0 = __byte_perm(w[4 * h], w[4 * h + 1], 0x5140), t1 = __byte_perm(w[4 * h + 2], w[4 * h + 3], 0x5140);
+        const uint32_t t2 = __byte_perm(w[4 * h], w[4 * h + 1], 0x7362), t3 = __byte_perm(w[4 * h + 2], w[4 * h + 3], 0x7362);
+        o[0][h] = __byte_perm(t0, t1, 0x5410); o[1][h] = __byte_perm(t0, t1, 0x7632);
+        o[2][h] = __byte_perm(t2, t3, 0x5410); o[3][h] = __byte_perm(t2, t3, 0x7632);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) *reinterpret_cast<uint2*>(&tile[i * 32 + pq][cg * 8]) = make_uint2(o[i][0], o[i][1]);
     __syncthreads();
-    const int pix = t >> 2, cq = (t & 3) * 16;
-    if (p0 + pix < HW) {
-        if (c0 + cq + 16 <= C && (C & 15) == 0) {
-            *reinterpret_cast<uint4*>(dst + (size_t)(p0 + pix) * C + c0 + cq) = *reinterpret_cast<const uint4*>(&tile[pix][cq]);
+    const bool pieces = ((C & 15) == 0) && ((reinterpret_cast<uintptr_t>(out) & 15) == 0);
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const int idx = t + 256 * r;
+        const int pix = idx >> 2, cq = (idx & 3) * 16;
+        const int slot = (pix & 3) * 32 + (pix >> 2);
+        if (p0 + pix >= HW) continue;
+        if (pieces && c0 + cq + 16 <= C) {
+            *reinterpret_cast<uint4*>(dst + (size_t)(p0 + pix) * C + c0 + cq) = *reinterpret_cast<const uint4*>(&tile[slot][cq]);
         } else {
             for (int j = 0; j < 16; ++j)
-                if (c0 + cq + j < C) dst[(size_t)(p0 + pix) * C + c0 + cq + j] = (int8_t)tile[pix][cq + j];
+                if (c0 + cq + j < C) dst[(size_t)(p0 + pix) * C + c0 + cq + j] = (int8_t)tile[slot][cq + j];
         }
     }
 }
@@ -216,7 +237,7 @@ int nq_conv_implicit_gemm(const int8_t* X, const void* Wt, int64_t ldw, int part
     const int8_t* x_nhwc = X;
     if (d->x_nchw) {
         const int HW = d->H * d->W;
-        dim3 grid((HW + 63) / 64, (d->Cin + 63) / 64, d->B);
+        dim3 grid((HW + 127) / 128, (d->Cin + 63) / 64, d->B);
         nchw_to_nhwc_kernel<<<grid, 256, 0, stream>>>(X, (int8_t*)workspace, d->Cin, HW);
         if (cudaGetLastError() != cudaSuccess) return NQ_ERR_CUDA;
         x_nhwc = (const int8_t*)workspace;
