@@ -50,10 +50,25 @@ struct ConvGeom {
     int tiles_w, tiles_h;
 };
 
+// Division by a number fixed at launch: q = (umulhi(n, magic) + n) >> shift, exact for n < 2^31 (magic = 0 for a
+// power of two).  The tile walk of every role divides twice per tile; the hardware's integer division cost the
+// epilogue warps about as much as one of their four output chunks.
+struct FastDiv {
+    uint32_t magic, shift;
+};
+inline FastDiv make_fastdiv(uint32_t d) {
+    FastDiv f{0u, 0u};
+    while ((1u << f.shift) < d) ++f.shift;
+    if ((1u << f.shift) != d) f.magic = (uint32_t)(((1ull << 32) * ((1ull << f.shift) - d)) / d + 1);
+    return f;
+}
+__device__ __forceinline__ uint32_t fast_div(uint32_t n, const FastDiv& f) { return (__umulhi(n, f.magic) + n) >> f.shift; }
+
 struct ContractionArgs {
     ConvGeom g;
     int M, N, K;
     int m_tiles, n_tiles, k_blocks;
+    FastDiv div_group, div_last;   // by kGroupM * n_tiles, and by the row count of the last (short) group of M-tiles
     const float* w_scale;
     const float* bias;
     float act_scale;
@@ -101,14 +116,19 @@ __host__ __device__ inline int contraction_smem_bytes(int bn, bool part, int h_b
     return bytes + 1024;                // slack to align the base to 1024 B
 }
 
-__device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, int& mt, int& nt) {
-    const int per_group = kGroupM * n_tiles;
-    const int g = tile / per_group;
+__device__ __forceinline__ void tile_coords(int tile, const ContractionArgs& p, int& mt, int& nt) {
+    const int per_group = kGroupM * p.n_tiles;
+    const int g = (int)fast_div((uint32_t)tile, p.div_group);
     const int first = g * kGroupM;
-    const int gsz = min(m_tiles - first, kGroupM);
     const int local = tile - g * per_group;
-    mt = first + local % gsz;
-    nt = local / gsz;
+    if (p.m_tiles - first >= kGroupM) {                  // a full group: kGroupM is a power of two
+        mt = first + (local & (kGroupM - 1));
+        nt = local / kGroupM;
+    } else {
+        const int gsz = p.m_tiles - first;
+        nt = (int)fast_div((uint32_t)local, p.div_last);
+        mt = first + local - nt * gsz;
+    }
 }
 
 // One 32-element unit of packed H-bit fields as it sits in the shared-memory tile ...
@@ -535,7 +555,7 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
                 int mt, nt;
-                tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
+                tile_coords(tile, p, mt, nt);
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
                     const uint32_t s = it % STAGES, use = it / STAGES;
                     if (!(ok = mbar_wait(smem_u32(&empty[s]), (use & 1) ^ 1, abort_flag, p.status, 0x10u))) break;
@@ -580,7 +600,7 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
                 int mt, nt;
-                tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
+                tile_coords(tile, p, mt, nt);
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++pit) {
                     const uint32_t ps = pit % p.packed_stages, puse = pit / p.packed_stages;
                     if (!(ok = mbar_wait(smem_u32(&pempty[ps]), (puse & 1) ^ 1, abort_flag, p.status, 0x11u))) break;
@@ -645,7 +665,7 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                              ((reinterpret_cast<uintptr_t>(p.acc_out) & 15) == 0);
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tl) {
             int mt, nt;
-            tile_coords(tile, p.m_tiles, p.n_tiles, mt, nt);
+            tile_coords(tile, p, mt, nt);
             const uint32_t buf = tl & 1, buse = tl >> 1;
             const int n0 = nt * BN;
             // per-channel factor: fl(fl(act * w_scale) * 2^l), then the exact 2^-(8-h) of the unpack.
@@ -668,7 +688,7 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             float sc_n[SCALES_PER_LANE], bs_n[SCALES_PER_LANE];
             if (tile + (int)gridDim.x < num_tiles) {
                 int mt_n;
-                tile_coords(tile + (int)gridDim.x, p.m_tiles, p.n_tiles, mt_n, next_nt);
+                tile_coords(tile + (int)gridDim.x, p, mt_n, next_nt);
                 if (next_nt != nt) fetch_scales<SCALES_PER_LANE>(p, next_nt * BN + chalf * (BN / 2), lane, sc_n, bs_n);
             }
             ok = mbar_wait(smem_u32(&tfull[buf]), buse & 1, abort_flag, p.status, 0x30u);

@@ -86,7 +86,7 @@ template <int H>
 __device__ __forceinline__ void fetch_stage(const ContractionArgs& p, const PairUnpackCtx& cx, const StageCursor& c,
                                             PackedUnit (&raw)[kPairUnitsPerThread]) {
     int mt2, nt;
-    tile_coords(c.tile, p.m_tiles, p.n_tiles, mt2, nt);
+    tile_coords(c.tile, p, mt2, nt);
     const int brow = nt * kPairBN + (int)cx.rank * (kPairBN / 2);
     const uint8_t* base = p.packed_b + (long long)c.kb * (16 * H);
 #pragma unroll
@@ -210,7 +210,7 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             bool ok = true;
             for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
                 int mt2, nt;
-                tile_coords(tile, p.m_tiles, p.n_tiles, mt2, nt);
+                tile_coords(tile, p, mt2, nt);
                 const int mt = mt2 * 2 + (int)rank;            // this CTA's 128-row tile
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
                     const uint32_t s = it % STAGES, use = it / STAGES;
@@ -256,7 +256,7 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             bool ok = true;
             for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
                 int mt2, nt;
-                tile_coords(tile, p.m_tiles, p.n_tiles, mt2, nt);
+                tile_coords(tile, p, mt2, nt);
                 const int brow = nt * BN + (int)rank * HALF;
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++pit) {
                     const uint32_t ps = pit % p.packed_stages, puse = pit / p.packed_stages;
@@ -326,7 +326,7 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         float* bs_w = sBias + (warp - 2) * (BN / 2);
         for (int tile = pair; ok && tile < num_tiles; tile += num_pairs, ++tl) {
             int mt2, nt;
-            tile_coords(tile, p.m_tiles, p.n_tiles, mt2, nt);
+            tile_coords(tile, p, mt2, nt);
             const int mt = mt2 * 2 + (int)rank;
             const uint32_t buf = tl & 1, buse = tl >> 1;
             const int n0 = nt * BN;
@@ -346,7 +346,7 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             float sc_n[SCALES_PER_LANE], bs_n[SCALES_PER_LANE];
             if (tile + num_pairs < num_tiles) {
                 int mt_n;
-                tile_coords(tile + num_pairs, p.m_tiles, p.n_tiles, mt_n, next_nt);
+                tile_coords(tile + num_pairs, p, mt_n, next_nt);
                 if (next_nt != nt) fetch_scales<SCALES_PER_LANE>(p, next_nt * BN + chalf * (BN / 2), lane, sc_n, bs_n);
             }
             ok = mbar_wait_cluster(smem_u32(&tfull[buf]), buse & 1, abort_flag, p.status, 0x130u);

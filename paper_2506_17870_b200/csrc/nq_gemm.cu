@@ -233,6 +233,8 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
     a.m_tiles = pair ? (m_tiles + 1) / 2 : m_tiles;
     a.n_tiles = (int)((N + bn - 1) / bn);
     a.k_blocks = k_blocks;
+    a.div_group = make_fastdiv((uint32_t)(kGroupM * a.n_tiles));
+    a.div_last = make_fastdiv((uint32_t)((a.m_tiles % kGroupM) ? (a.m_tiles % kGroupM) : 1));
     a.w_scale = w_scale; a.bias = bias; a.act_scale = act_scale;
     a.acc_out = acc_out; a.ld_acc = ld_acc; a.y = Y; a.ldy = ldy; a.y_is_bf16 = (y_dtype == NQ_BF16);
     a.status = status_word();
