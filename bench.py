@@ -44,6 +44,33 @@ METRIC = "nested_int8_gemm_tops"
 CONV_H = 6
 
 
+# DRAM bytes (read + written, MB) of one GEMM launch, from the ncu capture summarised in
+# profiles/gemm_dram_traffic_4096_8192.md (tile-store epilogue, 40 ns barrier probes).  16384 was not captured (over
+# a gigabyte per launch): it is taken as four times 8192, every operand and the output growing fourfold.  Must be set
+# to None again when the contraction kernels change.
+NCU_GEMM_DRAM_MB = {
+    4096: {4: 25.8, 5: 28.0, 6: 30.2, 7: 32.4, 0: 34.9},
+    8192: {4: 255.0, 5: 283.0, 6: 314.0, 7: 340.0, 0: 352.0},
+}
+
+
+def gemm_traffic_bytes_per_launch(sizes):
+    """Mean DRAM traffic of the GEMM launches of one step (h = 4..7 part-bit + one full-bit per size), or None."""
+    if NCU_GEMM_DRAM_MB is None:
+        return None
+    total, n = 0.0, 0
+    for s in sizes:
+        table, factor = NCU_GEMM_DRAM_MB.get(s), 1.0
+        if table is None and s == 16384:
+            table, factor = NCU_GEMM_DRAM_MB.get(8192), 4.0
+        if table is None:
+            return None
+        for h in list(HS) + [0]:
+            total += table[h] * factor * 1e6
+            n += 1
+    return total / n
+
+
 def measured_peaks():
     p = ROOT / "MEASURED_PEAKS.json"
     if p.exists():
@@ -296,7 +323,10 @@ def run_ours(args, rank, world, local_rank):
         "achieved": round(achieved, 1), "peak": round(int8_peak, 1), "unit": "TOP/s",
         "frac": round(achieved / int8_peak, 4),
         "peak_source": "2 x the %s bf16 burst figure (dense INT8 : bf16 nominal ratio 4.5 : 2.25)" % peaks["source"],
-        "launches": gemm_n, "avg_launch_ms": round(gemm_ms / max(gemm_n, 1), 4), "traffic": None,
+        "launches": gemm_n, "avg_launch_ms": round(gemm_ms / max(gemm_n, 1), 4),
+        "traffic": gemm_traffic_bytes_per_launch(sizes),
+        "traffic_unit": "DRAM bytes per launch, mean over the step's GEMM launches (ncu, profiles/gemm_dram_traffic_4096_8192.md)",
+        "algorithmic_bytes_per_launch": float(np.mean([s * s * (1 + (h / 8.0 if h else 1.0) + 2) for s in sizes for h in list(HS) + [0]])),
     }
     conv_note = (", + config 2: the ResNet-18-shaped stack (%d layers), batch %d, NCHW int8 in, both modes"
                  % (len(conv_layers), args.conv_batch) if have_conv else "")
