@@ -9,7 +9,7 @@
 //
 // Roles per CTA are those of the single-CTA kernel (nq_contraction.cuh): warp 0 TMA producer, warp 1 MMA
 // issuer (only in the even, "leader" CTA; it also owns the TMEM allocation in both), warps 2-9 epilogue,
-// warps 10-17 unpackers (part-bit).  Barrier protocol, all barriers at the same offsets in both CTAs:
+// warps 10-17 unpackers (part-bit), warp 18 producer of the packed-tile ring (part-bit, ring variant).  Barrier protocol, all barriers at the same offsets in both CTAs:
 //   full[s]    lives in the leader: 1 arrival by the leader's producer, which announces the bytes of BOTH
 //              CTAs' loads; the partner's loads complete on it through its cluster address.  In part-bit
 //              mode the leader's unpack warps arrive on it, and each of the partner's unpack warps sends it
@@ -133,8 +133,15 @@ __device__ __forceinline__ void pair_unpack_direct(const ContractionArgs& p, con
     }
 }
 
+// The ring variant of part-bit gives the packed-tile producer a warp of its own (the last one): two producers
+// that spin in one warp hold each other up for the length of a barrier probe.
+constexpr int kPackedProducerWarp = kFirstUnpackWarp + kUnpackWarps;
+__host__ __device__ constexpr int pair_threads(bool part, bool direct) {
+    return part ? (direct ? kBaseThreads + kUnpackThreads : kBaseThreads + kUnpackThreads + 32) : kBaseThreads;
+}
+
 template <bool PART, int MODE, bool DIRECT = false>
-__global__ void __launch_bounds__(PART ? kBaseThreads + kUnpackThreads : kBaseThreads, 1)
+__global__ void __launch_bounds__(pair_threads(PART, DIRECT), 1)
 contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                         const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmAcc,
                         const ContractionArgs p) {
@@ -249,7 +256,9 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                 const long long t0 = clock64();                // let copies in flight land before shared memory is released
                 while (clock64() - t0 < (1ll << 22)) { }
             }
-        } else if (PART && !DIRECT && lane == 1) {
+        }
+    } else if (PART && !DIRECT && warp == kPackedProducerWarp) {
+        if (lane == 0) {
             // ---- packed-tile producer: runs ahead of the A loads by up to the depth of its own ring, which
             //      is what hides the latency of fetching the weights
             uint32_t pit = 0;
@@ -410,7 +419,7 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             case 3: pair_unpack_direct<MODE, 3>(p, cx); break;
             default: pair_unpack_direct<MODE, 4>(p, cx); break;
         }
-    } else if (PART) {
+    } else if (PART && warp < kPackedProducerWarp) {
         // ------------------------------------------------------------------ unpackers (both CTAs, own half of B)
         const int group = (warp - kFirstUnpackWarp) / kUnpackGroupWarps;
         const int utid = (threadIdx.x - kBaseThreads) % kUnpackGroupThreads;

@@ -128,7 +128,7 @@ int launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const OutMaps& o
     const int pairs = tiles < max_pairs ? tiles : max_pairs;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * pairs, 1, 1);
-    cfg.blockDim = dim3(PART ? kBaseThreads + kUnpackThreads : kBaseThreads, 1, 1);
+    cfg.blockDim = dim3(pair_threads(PART, DIRECT), 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
