@@ -483,8 +483,15 @@ __device__ __forceinline__ void fetch_scales(const ContractionArgs& p, int col_b
     }
 }
 
+// Part-bit blocks end with one more warp, the producer of the packed-tile ring: two producers that spin in one
+// warp hold each other up for the length of a barrier probe.
+constexpr int kPackedProducerWarp = kFirstUnpackWarp + kUnpackWarps;
+__host__ __device__ constexpr int contraction_threads(bool part) {
+    return part ? kBaseThreads + kUnpackThreads + 32 : kBaseThreads;
+}
+
 template <int BN, bool PART, int MODE>
-__global__ void __launch_bounds__(PART ? kBaseThreads + kUnpackThreads : kBaseThreads, 1)
+__global__ void __launch_bounds__(contraction_threads(PART), 1)
 contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                    const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmAcc,
                    const ContractionArgs p) {
@@ -593,7 +600,9 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 const long long t0 = clock64();
                 while (clock64() - t0 < (1ll << 22)) { }
             }
-        } else if (PART && lane == 1) {
+        }
+    } else if (PART && warp == kPackedProducerWarp) {
+        if (lane == 0) {
             // ---- packed-tile producer: runs ahead of the A loads by up to the depth of its own ring, which
             //      is what hides the latency of fetching the weights
             uint32_t pit = 0;
@@ -736,8 +745,8 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             }
         }
         if (lane == 0) bulk_wait_all();                    // this lane's tile stores are done before the block leaves
-    } else if (PART) {
-        // ------------------------------------------------------------------ unpackers (warps 6-13)
+    } else if (PART && warp < kPackedProducerWarp) {
+        // ------------------------------------------------------------------ unpackers
         const int utid = threadIdx.x - kBaseThreads;
         uint32_t it = 0;
         bool ok = true;

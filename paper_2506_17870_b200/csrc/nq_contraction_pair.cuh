@@ -135,7 +135,6 @@ __device__ __forceinline__ void pair_unpack_direct(const ContractionArgs& p, con
 
 // The ring variant of part-bit gives the packed-tile producer a warp of its own (the last one): two producers
 // that spin in one warp hold each other up for the length of a barrier probe.
-constexpr int kPackedProducerWarp = kFirstUnpackWarp + kUnpackWarps;
 __host__ __device__ constexpr int pair_threads(bool part, bool direct) {
     return part ? (direct ? kBaseThreads + kUnpackThreads : kBaseThreads + kUnpackThreads + 32) : kBaseThreads;
 }

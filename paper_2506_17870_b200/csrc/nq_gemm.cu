@@ -97,7 +97,7 @@ int launch(const CUtensorMap& tmA, const CUtensorMap& tmB, const OutMaps& om, co
     }
     const int tiles = a.m_tiles * a.n_tiles;
     const int grid = tiles < sm_count() ? tiles : sm_count();
-    contraction_kernel<BN, PART, MODE><<<grid, PART ? kBaseThreads + kUnpackThreads : kBaseThreads, smem, stream>>>(tmA, tmB, om.y, om.acc, a);
+    contraction_kernel<BN, PART, MODE><<<grid, contraction_threads(PART), smem, stream>>>(tmA, tmB, om.y, om.acc, a);
     return cudaGetLastError() == cudaSuccess ? NQ_OK : NQ_ERR_CUDA;
 }
 
