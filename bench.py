@@ -45,12 +45,12 @@ CONV_H = 6
 
 
 # DRAM bytes (read + written, MB) of one GEMM launch, from the ncu capture summarised in
-# profiles/gemm_dram_traffic_4096_8192.md (tile-store epilogue, 40 ns barrier probes).  16384 was not captured (over
+# profiles/gemm_dram_traffic_4096_8192.md (tile-store epilogue, 40 ns barrier probes, packed-tile producer warp).  16384 was not captured (over
 # a gigabyte per launch): it is taken as four times 8192, every operand and the output growing fourfold.  Must be set
 # to None again when the contraction kernels change.
 NCU_GEMM_DRAM_MB = {
-    4096: {4: 25.8, 5: 28.0, 6: 30.2, 7: 32.4, 0: 34.9},
-    8192: {4: 255.0, 5: 283.0, 6: 314.0, 7: 340.0, 0: 352.0},
+    4096: {4: 26.5, 5: 27.8, 6: 30.1, 7: 32.2, 0: 34.3},
+    8192: {4: 270.0, 5: 288.0, 6: 311.0, 7: 342.0, 0: 356.0},
 }
 
 
