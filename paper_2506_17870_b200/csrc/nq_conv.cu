@@ -113,33 +113,54 @@ __global__ void __launch_bounds__(256) im2col_kernel(const int8_t* __restrict__ 
 
 // The same patch matrix for layers with few input channels (the stem): one block per output row (b, p).  The
 // R input rows it needs are staged in shared memory for all channels with the padding columns already
-// zero, and a small table gives, for every k, where its byte sits relative to the patch origin; each output
+// zero (NCHW rows are copied word by word), and a small table gives, for every k, where its byte sits relative to the patch origin; each output
 // byte is then two shared-memory reads, and whole 16-byte chunks go out coalesced.
 __global__ void __launch_bounds__(256) im2col_rows_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ a,
                                                           nq_conv_desc d, int Ho, int Wo, int K, int ld) {
     extern __shared__ uint8_t sm[];
-    const int Wp = d.W + 2 * d.pad;
-    uint8_t* patch = sm;                                           // [R][Cin][Wp]
-    uint16_t* lut = reinterpret_cast<uint16_t*>(sm + ((d.R * d.Cin * Wp + 15) & ~15));   // [ld]
+    // patch[r][ci][pitch]: a padded input row starts `shift` bytes into its slot, so that the first real pixel
+    // (after the left padding) sits on a 4-byte boundary and whole words of the input can be dropped in
+    const int shift = (4 - (d.pad & 3)) & 3;
+    const int pitch = (d.W + 2 * d.pad + shift + 3) & ~3;
+    const int rows = d.R * d.Cin;
+    uint8_t* patch = sm;
+    uint16_t* lut = reinterpret_cast<uint16_t*>(sm + ((rows * pitch + 15) & ~15));   // [ld]
     const int p = blockIdx.x, b = blockIdx.y;
-    for (int i = threadIdx.x; i < d.R * d.Cin * Wp; i += blockDim.x) {
-        const int col = i % Wp, rc = i / Wp;
-        const int ci = rc % d.Cin, r = rc / d.Cin;
-        const int ih = p * d.stride - d.pad + r, iw = col - d.pad;
-        uint8_t v = 0;
-        if (ih >= 0 && ih < d.H && iw >= 0 && iw < d.W) {
-            const size_t off = d.x_nchw ? (((size_t)b * d.Cin + ci) * d.H + ih) * d.W + iw
-                                        : (((size_t)b * d.H + ih) * d.W + iw) * d.Cin + ci;
-            v = (uint8_t)x[off];
+    const bool words = d.x_nchw && ((d.W & 3) == 0) && ((reinterpret_cast<uintptr_t>(x) & 3) == 0);
+    if (words) {
+        // zero everything (padding columns, rows above and below the image), then copy the rows word by word:
+        // 64 threads walk a row, four rows at a time -- no division anywhere
+        for (int i = threadIdx.x; i < rows * pitch / 4; i += blockDim.x) reinterpret_cast<uint32_t*>(patch)[i] = 0u;
+        __syncthreads();
+        const int wpr = d.W >> 2;
+        for (int rc = threadIdx.x >> 6; rc < rows; rc += blockDim.x >> 6) {
+            const int r = rc / d.Cin, ci = rc - r * d.Cin;
+            const int ih = p * d.stride - d.pad + r;
+            if (ih < 0 || ih >= d.H) continue;
+            const uint32_t* src = reinterpret_cast<const uint32_t*>(x + (((size_t)b * d.Cin + ci) * d.H + ih) * d.W);
+            uint32_t* dst = reinterpret_cast<uint32_t*>(patch + rc * pitch + shift + d.pad);
+            for (int wc = threadIdx.x & 63; wc < wpr; wc += 64) dst[wc] = __ldg(src + wc);
         }
-        patch[i] = v;
+    } else {
+        for (int i = threadIdx.x; i < rows * pitch; i += blockDim.x) {
+            const int col = i % pitch - shift, rc = i / pitch;
+            const int ci = rc % d.Cin, r = rc / d.Cin;
+            const int ih = p * d.stride - d.pad + r, iw = col - d.pad;
+            uint8_t v = 0;
+            if (ih >= 0 && ih < d.H && iw >= 0 && iw < d.W) {
+                const size_t off = d.x_nchw ? (((size_t)b * d.Cin + ci) * d.H + ih) * d.W + iw
+                                            : (((size_t)b * d.H + ih) * d.W + iw) * d.Cin + ci;
+                v = (uint8_t)x[off];
+            }
+            patch[i] = v;
+        }
     }
     for (int k = threadIdx.x; k < ld; k += blockDim.x) {
         uint16_t o = 0xffffu;                                      // beyond K: zero
         if (k < K) {
             const int tap = k / d.Cin, ci = k - tap * d.Cin;
             const int r = tap / d.S, s = tap - r * d.S;
-            o = (uint16_t)((r * d.Cin + ci) * Wp + s);
+            o = (uint16_t)((r * d.Cin + ci) * pitch + shift + s);
         }
         lut[k] = o;
     }
@@ -219,8 +240,9 @@ int nq_conv_implicit_gemm(const int8_t* X, const void* Wt, int64_t ldw, int part
         // explicit patch matrix, then the plain GEMM path
         const int ld = (int)((K + 15) / 16 * 16);
         const long long chunks = M * (ld / 16);
-        const size_t rows_smem = (((size_t)d->R * d->Cin * (d->W + 2 * d->pad) + 15) & ~size_t(15)) + (size_t)ld * 2;
-        if (rows_smem <= 48 * 1024 && (size_t)d->R * d->Cin * (d->W + 2 * d->pad) + (size_t)Wo * d->stride < 0xffff &&
+        const size_t row_pitch = ((size_t)d->W + 2 * d->pad + ((4 - (d->pad & 3)) & 3) + 3) & ~size_t(3);
+        const size_t rows_smem = (((size_t)d->R * d->Cin * row_pitch + 15) & ~size_t(15)) + (size_t)ld * 2;
+        if (rows_smem <= 48 * 1024 && (size_t)d->R * d->Cin * row_pitch + (size_t)Wo * d->stride < 0xffff &&
             Ho <= 65535 * 32 && d->B <= 65535) {
             im2col_rows_kernel<<<dim3(Ho, d->B), 256, rows_smem, stream>>>(X, (int8_t*)workspace, *d, Ho, Wo, (int)K, ld);
         } else {
