@@ -166,6 +166,14 @@ def test_tile_stores_and_plain_stores_agree(M, N, K, bf16, monkeypatch):
                                                   y2.view(torch.int16 if bf16 else torch.int32))
 
 
+@pytest.mark.parametrize("M,N,K", [(200, 8, 64), (33, 16, 128), (129, 4, 32)])
+def test_outputs_narrower_than_a_store_box(M, N, K):
+    """Output rows shorter than the 64-byte box of a tile store (aligned pitch, so the tile-store path is taken)."""
+    d = wl.gemm_inputs(91, M + N + K, M, N, K)
+    run_both_modes(d, 8, 6)
+    run_both_modes(d, 8, 6, bf16=True)
+
+
 @pytest.mark.parametrize("size,h", [(4096, 6), (4096, 4)])
 def test_large_square_gemm_sampled_rows_and_checksums(size, h):
     """Config-4 shape in the launch configuration the benchmark times: sampled rows bit-exact
