@@ -348,6 +348,7 @@ def run_ours(args, rank, world, local_rank):
     }
     if model_switch is not None:
         line["rows"]["model_switch"] = model_switch
+        line["rows"]["word64_convert_8192"] = _word64_rows(nq, torch, dev)
     if model_rows is not None:
         line["rows"].update(model_rows)
     if world == 1 and not args.no_cpu_baseline:
@@ -438,6 +439,40 @@ def _model_switch(nq, torch, wl, dev):
         res["tensors"] = len(shapes)
         res["algorithmic_mb"] = round(nbytes / 1e6, 1)
         out[name] = res
+    return out
+
+
+def _word64_rows(nq, torch, dev):
+    """The paper's packed-bit tensors (64 // k fields per 64-bit word) converted to the sliced layout and back on the
+    device: one 8192 x 8192 tensor per field width, bytes read + written over the median of 5 launches."""
+    peaks = measured_peaks()
+    out = {}
+    rows = cols = 8192
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(7)
+    for bits in (4, 5, 6):
+        lim = 1 << (bits - 1)
+        v = torch.randint(-lim, lim, (rows, cols), dtype=torch.int8, device=dev, generator=gen)
+        sliced = nq.nq_pack(v, bits)
+        words = nq.nq_sliced_to_word64(sliced, bits, rows, cols)
+        nbytes = sliced.numel() + words.numel() * 8
+        row = {}
+        for name, fn in (("to_sliced", lambda: nq.nq_word64_to_sliced(words, bits, cols)),
+                         ("to_word64", lambda: nq.nq_sliced_to_word64(sliced, bits, rows, cols))):
+            ts = []
+            for rep in range(6):
+                a = torch.cuda.Event(enable_timing=True)
+                b = torch.cuda.Event(enable_timing=True)
+                a.record()
+                fn()
+                b.record()
+                torch.cuda.synchronize()
+                if rep:
+                    ts.append(a.elapsed_time(b))
+            ms = float(np.median(ts))
+            g = nbytes / (ms * 1e-3) / 1e9
+            row[name] = {"us": round(ms * 1e3, 1), "gbs": round(g, 0), "frac_hbm": round(g / peaks["hbm_gbs"], 3)}
+        out[f"k{bits}"] = row
     return out
 
 

@@ -110,6 +110,20 @@ NQ_API int nq_pack(const int8_t *values, int64_t ld, int bits, int64_t rows, int
             void *packed_out, void *stream);
 
 /*
+ * The paper's packed-bit tensor ("Deployment": nested weights are stored as packed-bit tensors in unsigned
+ * INT64 words, e.g. twenty-one 3-bit or twelve 5-bit weights per word) and conversion to and from the sliced
+ * layout, on the device.  A [rows, cols] tensor of k-bit fields takes nq_word64_row_words(cols, k) words per
+ * row, rows dense; word w of a row holds the fields of elements w * (64 / k) ... in order, field j at bits
+ * [j * k, j * k + k), two's complement, unused top bits and fields past `cols` zero.  (The paper fixes the count
+ * per word; the order of the fields inside a word is this library's reading.)
+ *   words (device)  uint64, 8-byte aligned;  packed (device)  sliced tensor, 16-byte aligned
+ * nq_word64_row_words returns -1 on bad arguments.
+ */
+NQ_API int64_t nq_word64_row_words(int64_t cols, int bits);
+NQ_API int nq_word64_to_sliced(const uint64_t *words, int bits, int64_t rows, int64_t cols, void *packed_out, void *stream);
+NQ_API int nq_sliced_to_word64(const void *packed, int bits, int64_t rows, int64_t cols, uint64_t *words_out, void *stream);
+
+/*
  * Whole-model page-in / page-out in ONE launch.  A model is a list of tensors; the caller builds
  * the list once with nq_batch_plan and then switches the model with a single call.
  *   descs (host)   count entries

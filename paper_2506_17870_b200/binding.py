@@ -25,6 +25,7 @@ NQ_F32, NQ_BF16 = 0, 1
 EXPORTS = (
     "nq_status_str", "nq_low_bits", "nq_packed_row_bytes", "nq_packed_bytes",
     "nq_decompose", "nq_recompose", "nq_drop_low", "nq_unpack", "nq_pack",
+    "nq_word64_row_words", "nq_word64_to_sliced", "nq_sliced_to_word64",
     "nq_batch_table_bytes", "nq_batch_plan", "nq_recompose_batched", "nq_drop_low_batched",
     "nq_gemm_full", "nq_gemm_part", "nq_conv_workspace_bytes", "nq_conv_implicit_gemm",
     "nq_conv_implicit_gemm_static",
@@ -65,7 +66,8 @@ def lib() -> ctypes.CDLL:
         except OSError as e:  # pragma: no cover
             raise NqLibraryError(f"cannot load {_LIB_PATH}: {e}") from e
         L.nq_status_str.restype = ctypes.c_char_p
-        for name in ("nq_packed_row_bytes", "nq_packed_bytes", "nq_batch_table_bytes", "nq_conv_workspace_bytes"):
+        for name in ("nq_packed_row_bytes", "nq_packed_bytes", "nq_batch_table_bytes", "nq_conv_workspace_bytes",
+                     "nq_word64_row_words"):
             getattr(L, name).restype = ctypes.c_int64
         _lib = L
     return _lib
@@ -181,6 +183,31 @@ def nq_pack(values: torch.Tensor, bits: int) -> torch.Tensor:
     out = _empty_packed(rows, cols, bits, values.device)
     _check(lib().nq_pack(_ptr(values), _i64(_ld(values)), bits, _i64(rows), _i64(cols), _ptr(out), _stream()),
            "nq_pack")
+    return out
+
+
+def nq_word64_row_words(cols: int, bits: int) -> int:
+    return int(lib().nq_word64_row_words(_i64(cols), bits))
+
+
+def nq_word64_to_sliced(words: torch.Tensor, bits: int, cols: int) -> torch.Tensor:
+    """[rows, nq_word64_row_words(cols, bits)] int64 words (the paper's packed-bit tensor) -> sliced tensor."""
+    _need(words, torch.int64, "words", 2)
+    rows = words.shape[0]
+    if not words.is_contiguous() or words.shape[1] != nq_word64_row_words(cols, bits):
+        raise ValueError("words must be a dense [rows, nq_word64_row_words(cols, bits)] tensor")
+    out = _empty_packed(rows, cols, bits, words.device)
+    _check(lib().nq_word64_to_sliced(_ptr(words), bits, _i64(rows), _i64(cols), _ptr(out), _stream()), "nq_word64_to_sliced")
+    return out
+
+
+def nq_sliced_to_word64(packed: torch.Tensor, bits: int, rows: int, cols: int) -> torch.Tensor:
+    """Sliced tensor -> [rows, nq_word64_row_words(cols, bits)] int64 words."""
+    _need(packed, torch.uint8, "packed")
+    if packed.numel() != nq_packed_bytes(rows, cols, bits):
+        raise ValueError("packed has the wrong size for (rows, cols, bits)")
+    out = torch.empty((rows, nq_word64_row_words(cols, bits)), dtype=torch.int64, device=packed.device)
+    _check(lib().nq_sliced_to_word64(_ptr(packed), bits, _i64(rows), _i64(cols), _ptr(out), _stream()), "nq_sliced_to_word64")
     return out
 
 

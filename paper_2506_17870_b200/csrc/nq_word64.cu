@@ -1,0 +1,173 @@
+// Converters between the paper's packed-bit tensor and the library's sliced layout.
+//
+// The paper ("Deployment": packed-bit tensors) stores a k-bit weight tensor as unsigned 64-bit words with
+// 64 // k fields each, field j at bits [j*k, j*k + k), the unused top bits zero (twenty-one 3-bit or twelve
+// 5-bit weights per word).  That is the format a model arrives in; the kernels of this library work on the
+// sliced layout of nq.h.  Both directions are plain element-wise moves of k-bit two's-complement fields:
+//   word64 -> sliced   one thread per 32-element unit: walks the words that hold its fields, then lays the
+//                      unit's slices down word by word
+//   sliced -> word64   one thread per output word: gathers its 64 // k fields out of the slices
+// They are conversion utilities (run once per model), written for clarity; the hot codec is nq_codec.cu.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/nq.h"
+#include "nq_internal.cuh"
+
+namespace {
+
+// Where slice `s` (a power of two) keeps the bits of group element e: byte offset inside the slice and shift
+// inside that byte (the first of the 8/s fields that share a byte sits in its top bits).
+__device__ __forceinline__ void slice_place(int s, int e, int& byte_off, int& shift) {
+    const int unit = e >> 5, q = (e & 31) >> 2, lane = e & 3;
+    const int per_byte = 8 / s;
+    const int word = q / per_byte, sub = q - word * per_byte;
+    byte_off = ((unit * s + word) << 2) + lane;
+    shift = 8 - s * sub - s;
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(256) word64_to_sliced_kernel(const uint64_t* __restrict__ words, int64_t rows,
+                                                               int64_t cols, uint8_t* __restrict__ packed) {
+    constexpr int PER = 64 / BITS;
+    constexpr uint64_t MASK = (1ull << BITS) - 1ull;
+    const int64_t units_per_row = ((cols + 127) >> 7) << 2;
+    const int64_t row_words = (cols + PER - 1) / PER;
+    const int64_t total = rows * units_per_row;
+    for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < total; u += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = u / units_per_row, ur = u - row * units_per_row;
+        const int64_t c0 = ur * 32;
+        const uint64_t* wrow = words + row * row_words;
+        // the unit's 32 fields, read in order: the word index and the position inside the word advance together
+        uint32_t f[32];
+        int64_t wi = c0 / PER;
+        int fi = (int)(c0 - wi * PER);
+        uint64_t w = (c0 < cols) ? wrow[wi] : 0ull;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            f[j] = (c0 + j < cols) ? (uint32_t)((w >> (fi * BITS)) & MASK) : 0u;
+            if (++fi == PER) {
+                fi = 0;
+                ++wi;
+                w = (c0 + j + 1 < cols) ? wrow[wi] : 0ull;
+            }
+        }
+        uint8_t* group = packed + (row * (units_per_row >> 2) + (ur >> 2)) * 16 * BITS;
+        const int unit = (int)(ur & 3);
+        int used = 0, slice_base = 0;
+#pragma unroll
+        for (int s = 8; s >= 1; s >>= 1) {
+            if (!(BITS & s)) continue;
+            const int per_byte = 8 / s;
+#pragma unroll
+            for (int wq = 0; wq < s; ++wq) {
+                uint32_t out = 0;
+#pragma unroll
+                for (int sub = 0; sub < per_byte; ++sub) {
+                    const int q = wq * per_byte + sub;
+#pragma unroll
+                    for (int lane = 0; lane < 4; ++lane) {
+                        const uint32_t part = (f[q * 4 + lane] >> (BITS - used - s)) & ((1u << s) - 1u);
+                        out |= part << ((8 - s * sub - s) + 8 * lane);
+                    }
+                }
+                *reinterpret_cast<uint32_t*>(group + slice_base + ((unit * s + wq) << 2)) = out;
+            }
+            slice_base += 16 * s;
+            used += s;
+        }
+    }
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(256) sliced_to_word64_kernel(const uint8_t* __restrict__ packed, int64_t rows,
+                                                               int64_t cols, uint64_t* __restrict__ words) {
+    constexpr int PER = 64 / BITS;
+    const int64_t groups_per_row = (cols + 127) >> 7;
+    const int64_t row_words = (cols + PER - 1) / PER;
+    const int64_t total = rows * row_words;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = i / row_words, wd = i - row * row_words;
+        uint64_t out = 0;
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            const int64_t c = wd * PER + j;
+            if (c >= cols) break;
+            const uint8_t* group = packed + (row * groups_per_row + (c >> 7)) * 16 * BITS;
+            const int e = (int)(c & 127);
+            uint32_t field = 0;
+            int slice_base = 0;
+#pragma unroll
+            for (int s = 8; s >= 1; s >>= 1) {
+                if (!(BITS & s)) continue;
+                int off, sh;
+                slice_place(s, e, off, sh);
+                field = (field << s) | ((uint32_t)(group[slice_base + off] >> sh) & ((1u << s) - 1u));
+                slice_base += 16 * s;
+            }
+            out |= (uint64_t)field << (j * BITS);
+        }
+        words[i] = out;
+    }
+}
+
+inline int blocks_for(int64_t threads) {
+    const int64_t need = (threads + 255) / 256;
+    const int64_t cap = (int64_t)nq::sm_count() * 16;
+    return (int)(need < cap ? need : cap);
+}
+
+template <int BITS>
+int launch_bits(bool to_sliced, const void* src, int64_t rows, int64_t cols, void* dst, cudaStream_t s) {
+    if (to_sliced) {
+        const int64_t units = rows * (((cols + 127) >> 7) << 2);
+        word64_to_sliced_kernel<BITS><<<blocks_for(units), 256, 0, s>>>(static_cast<const uint64_t*>(src), rows, cols,
+                                                                       static_cast<uint8_t*>(dst));
+    } else {
+        const int64_t n = rows * ((cols + 64 / BITS - 1) / (64 / BITS));
+        sliced_to_word64_kernel<BITS><<<blocks_for(n), 256, 0, s>>>(static_cast<const uint8_t*>(src), rows, cols,
+                                                                    static_cast<uint64_t*>(dst));
+    }
+    return cudaGetLastError() == cudaSuccess ? NQ_OK : NQ_ERR_CUDA;
+}
+
+int convert(bool to_sliced, const void* src, int bits, int64_t rows, int64_t cols, void* dst, void* stream) {
+    if (rows < 0 || cols < 0) return NQ_ERR_INVALID_ARG;
+    if (bits < 1 || bits > 8) return NQ_ERR_UNSUPPORTED;
+    if (rows == 0 || cols == 0) return NQ_OK;
+    if (!src || !dst) return NQ_ERR_INVALID_ARG;
+    const void* sliced = to_sliced ? dst : src;
+    const void* w64 = to_sliced ? src : dst;
+    if ((reinterpret_cast<uintptr_t>(sliced) & 15) || (reinterpret_cast<uintptr_t>(w64) & 7)) return NQ_ERR_ALIGNMENT;
+    cudaStream_t s = (cudaStream_t)stream;
+    switch (bits) {
+        case 1: return launch_bits<1>(to_sliced, src, rows, cols, dst, s);
+        case 2: return launch_bits<2>(to_sliced, src, rows, cols, dst, s);
+        case 3: return launch_bits<3>(to_sliced, src, rows, cols, dst, s);
+        case 4: return launch_bits<4>(to_sliced, src, rows, cols, dst, s);
+        case 5: return launch_bits<5>(to_sliced, src, rows, cols, dst, s);
+        case 6: return launch_bits<6>(to_sliced, src, rows, cols, dst, s);
+        case 7: return launch_bits<7>(to_sliced, src, rows, cols, dst, s);
+        default: return launch_bits<8>(to_sliced, src, rows, cols, dst, s);
+    }
+}
+
+}  // namespace
+
+extern "C" {
+
+int64_t nq_word64_row_words(int64_t cols, int bits) {
+    if (cols < 0 || bits < 1 || bits > 8) return -1;
+    const int64_t per = 64 / bits;
+    return (cols + per - 1) / per;
+}
+
+int nq_word64_to_sliced(const uint64_t* words, int bits, int64_t rows, int64_t cols, void* packed_out, void* stream) {
+    return convert(true, words, bits, rows, cols, packed_out, stream);
+}
+
+int nq_sliced_to_word64(const void* packed, int bits, int64_t rows, int64_t cols, uint64_t* words_out, void* stream) {
+    return convert(false, packed, bits, rows, cols, words_out, stream);
+}
+
+}  // extern "C"
