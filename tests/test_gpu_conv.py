@@ -27,6 +27,9 @@ def host(t):
 def run_layer(L, batch, seed, n=8, h=6, nchw=True, check_y=True):
     d = wl.conv_layer_inputs(71, seed, L, batch)
     X, W, mask, ws, sa = d["X"], d["W"], d["mask"], d["w_scale"], d["act_scale"]
+    if n < 8:                      # INTn nesting: INTn weights and n-bit activations in int8 containers
+        W = (W >> (8 - n)).astype(np.int8)
+        X = (X >> (8 - n)).astype(np.int8)
     wh, wlo = oracle.decompose(W, mask, n, h, True)
     K = L.K
     ldw = -(-K // 16) * 16
@@ -101,6 +104,15 @@ def test_tile_stores_and_plain_stores_agree(L, monkeypatch):
     acc2, y2, _ = nq.nq_conv_implicit_gemm(x, w_mat, desc, ws, 0.02, want_acc=True, y_dtype=torch.bfloat16)
     nq.nq_device_status()
     assert torch.equal(acc, acc2) and torch.equal(y.view(torch.int16), y2.view(torch.int16))
+
+
+@pytest.mark.parametrize("n,h", [(6, 3), (6, 4), (6, 5), (8, 3)])
+def test_int6_nesting_and_three_bit_high_part(n, h):
+    """INT6 nesting (6-bit weights and activations, h in {3, 4, 5}) and the 3-bit high part of INT8 nesting through
+    both convolution modes, both operating modes."""
+    run_layer(C("c64", 64, 10, 10, 64, 3, 3, 1, 1), 3, 30 + n + h, n=n, h=h)
+    run_layer(C("c128", 128, 9, 9, 96, 3, 3, 2, 1), 3, 40 + n + h, n=n, h=h)
+    run_layer(C("stem", 3, 20, 20, 32, 7, 7, 2, 3), 2, 50 + n + h, n=n, h=h)
 
 
 def test_pointwise_convolution_equals_the_gemm_entry_point():
