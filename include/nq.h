@@ -86,6 +86,19 @@ NQ_API int nq_decompose(const int8_t *w_int, const uint8_t *mask, int64_t rows, 
                  void *packed_high, void *packed_low, void *stream);
 
 /*
+ * Rounding masks of the baselines NestQuant is compared with ("Higher-Bit Weights: Integer Data Optimization" and
+ * its ablation; the rows of the "Nesting Numerical Errors" table): for nq_decompose's `mask` argument when no
+ * adaptive-rounding optimiser supplies one.
+ *   NQ_ROUND_DOWN     BitShift: always the floor (mask 0 everywhere)
+ *   NQ_ROUND_UP       always the ceiling (mask 1 everywhere; nq_decompose leaves exact multiples of 2^l alone)
+ *   NQ_ROUND_NEAREST  RTN: the nearer neighbour of w_int / 2^l, a tie going to the even one
+ *   w_int (device) int8 [rows, cols] pitch ld_w;  mask_out (device, out) uint8 0 / 1, [rows, cols] pitch ld_mask
+ */
+enum { NQ_ROUND_DOWN = 0, NQ_ROUND_UP = 1, NQ_ROUND_NEAREST = 2 };
+NQ_API int nq_rounding_mask(const int8_t *w_int, int64_t ld_w, int64_t rows, int64_t cols, int n_bits, int h_bits,
+                     int mode, uint8_t *mask_out, int64_t ld_mask, void *stream);
+
+/*
  * Recomposition / page-in -- Eq. 5 read as the upgrade of "Nesting Mechanism of Decomposed
  * Weights": w_int = clip_INTn(w_high * 2^l + w_low), a shift and an ADD of the sign-extended low
  * field.  Output int8 [rows, cols] with row pitch ld_out elements (device, out).

@@ -25,7 +25,7 @@ NQ_F32, NQ_BF16 = 0, 1
 EXPORTS = (
     "nq_status_str", "nq_low_bits", "nq_packed_row_bytes", "nq_packed_bytes",
     "nq_decompose", "nq_recompose", "nq_drop_low", "nq_unpack", "nq_pack",
-    "nq_word64_row_words", "nq_word64_to_sliced", "nq_sliced_to_word64",
+    "nq_word64_row_words", "nq_word64_to_sliced", "nq_sliced_to_word64", "nq_rounding_mask",
     "nq_batch_table_bytes", "nq_batch_plan", "nq_recompose_batched", "nq_drop_low_batched",
     "nq_gemm_full", "nq_gemm_part", "nq_conv_workspace_bytes", "nq_conv_implicit_gemm",
     "nq_conv_implicit_gemm_static",
@@ -184,6 +184,20 @@ def nq_pack(values: torch.Tensor, bits: int) -> torch.Tensor:
     _check(lib().nq_pack(_ptr(values), _i64(_ld(values)), bits, _i64(rows), _i64(cols), _ptr(out), _stream()),
            "nq_pack")
     return out
+
+
+NQ_ROUND_DOWN, NQ_ROUND_UP, NQ_ROUND_NEAREST = 0, 1, 2
+
+
+def nq_rounding_mask(w_int: torch.Tensor, n_bits: int, h_bits: int, mode: int) -> torch.Tensor:
+    """Rounding mask (uint8 0 / 1, same shape and pitch as w_int) of one of the baseline roundings."""
+    _need(w_int, torch.int8, "w_int", 2)
+    rows, cols = w_int.shape
+    ld = _ld(w_int)
+    buf = torch.empty((rows, ld), dtype=torch.uint8, device=w_int.device)
+    _check(lib().nq_rounding_mask(_ptr(w_int), _i64(ld), _i64(rows), _i64(cols), n_bits, h_bits, int(mode), _ptr(buf),
+                                  _i64(ld), _stream()), "nq_rounding_mask")
+    return buf[:, :cols]
 
 
 def nq_word64_row_words(cols: int, bits: int) -> int:
