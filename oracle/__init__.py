@@ -192,6 +192,22 @@ def dequant(acc, w_scale, act_scale: float, l_shift: int = 0, bias=None, want_re
     return y
 
 
+def requant(acc, w_scale, act_scale: float, l_shift: int, out_scale: float, bias=None, relu: bool = True):
+    """INT8 activations for the next layer from a layer's accumulators (the library's own definition, fp32)."""
+    acc = _c(acc, np.int32)
+    lead = acc.shape[:-1]
+    N = acc.shape[-1]
+    acc2 = acc.reshape(-1, N)
+    M = acc2.shape[0]
+    ws = _c(w_scale, np.float32)
+    assert ws.shape == (N,)
+    b = None if bias is None else _c(bias, np.float32)
+    q = np.empty((M, N), dtype=np.int8)
+    _load().nqo_requant(_p(acc2), _i64(N), _i64(M), _i64(N), _p(ws), ctypes.c_float(act_scale), int(l_shift),
+                        None if b is None else _p(b), int(bool(relu)), ctypes.c_float(out_scale), _p(q), _i64(N))
+    return q.reshape(*lead, N)
+
+
 def f32_to_bf16_bits(x):
     x = _c(x, np.float32)
     out = np.empty(x.shape, dtype=np.uint16)

@@ -333,6 +333,40 @@ void nqo_dequant(const int32_t *acc, int64_t ldacc, int64_t M, int64_t N,
         }
 }
 
+/* ------------------------------------------------------------------------- */
+/* O6b  requantisation of a layer's output to INT8 for the next layer.  The    */
+/*      paper quantises activations to 8 bits ("8-bit activations") with the   */
+/*      uniform quantiser of Eq. 1 and zero-point 0, but does not say how a    */
+/*      layer's output becomes the next layer's input: PARITY UNPINNED by the  */
+/*      paper; this is the library's own definition, in fp32, one rounding per */
+/*      operation, in this order:                                              */
+/*        v = dequantised output as in O6 (+ bias)                             */
+/*        v = max(v, 0)                       when relu                        */
+/*        t = fl(v * fl(1 / out_scale))                                        */
+/*        q = clip(round-half-even(t), -128, 127)          (Eq. 1 with Z = 0)  */
+/* ------------------------------------------------------------------------- */
+void nqo_requant(const int32_t *acc, int64_t ldacc, int64_t M, int64_t N,
+                 const float *w_scale, float act_scale, int l_shift, const float *bias,
+                 int relu, float out_scale, int8_t *q, int64_t ldq)
+{
+    const float pow2 = (float)(1 << l_shift);
+    volatile float inv = 1.0f / out_scale;
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t j = 0; j < N; ++j) {
+            volatile float sj = act_scale * w_scale[j];
+            volatile float scale = sj * pow2;
+            volatile float v = (float)acc[m * ldacc + j] * scale;
+            if (bias) { volatile float t = v + bias[j]; v = t; }
+            if (relu && v < 0.0f) v = 0.0f;
+            volatile float t = v * inv;
+            float r = nearbyintf(t);              /* default rounding mode: to nearest, ties to even */
+            if (r < -128.0f) r = -128.0f;
+            if (r > 127.0f) r = 127.0f;
+            q[m * ldq + j] = (int8_t)r;
+        }
+}
+
 /* fp32 -> bf16, round to nearest, ties to even (finite inputs) */
 void nqo_f32_to_bf16(const float *x, int64_t count, uint16_t *out)
 {
