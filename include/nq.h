@@ -212,6 +212,28 @@ NQ_API int nq_conv_implicit_gemm(const int8_t *X, const void *Wt, int64_t ldw, i
                           void *workspace, int64_t workspace_bytes, void *stream);
 
 /*
+ * The same three layers with a requantising epilogue: the output is the next layer's INT8 activations, so layers
+ * can be chained on the device and the output traffic is a quarter of fp32.  The paper quantises activations to
+ * 8 bits with the uniform quantiser of Eq. 1 (zero-point 0) but does not say how one layer's output becomes the
+ * next layer's input; this is the library's own definition (fp32, one rounding per operation):
+ *   v = the dequantised value of nq_gemm_full / nq_gemm_part (+ bias[j])
+ *   v = max(v, 0)                                   when relu != 0
+ *   q = clip(round_half_even(fl(v * fl(1 / out_scale))), -128, 127)
+ *   Yq (device, out) int8 [M, N] pitch ldyq (convolution: NHWC, dense).  out_scale > 0 is the activation scale of
+ *   the next layer (its act_scale).  The other arguments are those of the fp32 / bf16 entry points.
+ */
+NQ_API int nq_gemm_full_q8(const int8_t *X, int64_t ldx, const int8_t *W, int64_t ldw, const float *w_scale,
+                    float act_scale, const float *bias, float out_scale, int relu,
+                    int64_t M, int64_t N, int64_t K, int8_t *Yq, int64_t ldyq, void *stream);
+NQ_API int nq_gemm_part_q8(const int8_t *X, int64_t ldx, const void *packed_high, int n_bits, int h_bits,
+                    const float *w_scale, float act_scale, const float *bias, float out_scale, int relu,
+                    int64_t M, int64_t N, int64_t K, int8_t *Yq, int64_t ldyq, void *stream);
+NQ_API int nq_conv_implicit_gemm_q8(const int8_t *X, const void *Wt, int64_t ldw, int part_bit, int n_bits, int h_bits,
+                             const nq_conv_desc *desc, const float *w_scale, float act_scale, const float *bias,
+                             float out_scale, int relu, int8_t *Yq,
+                             void *workspace, int64_t workspace_bytes, void *stream);
+
+/*
  * The convolution again, for callers that must not allocate.  (The paper has no counterpart; this is a
  * convenience of the library.)  nq_conv_implicit_gemm needs a workspace whenever it re-lays the input
  * (NCHW activations, or a channel count it cannot gather in place), and somebody has to allocate that.

@@ -85,6 +85,9 @@ struct ContractionArgs {
     long long ldy;
     int y_is_bf16;
     int y_tma, acc_tma;  // the output is written with tile stores through tmY / tmAcc (aligned base and pitch)
+    int y_is_i8;         // requantised INT8 output: q = clip(rint(fl(relu(v) * inv_out_scale)))
+    int relu;
+    float inv_out_scale;
     unsigned int* status;
 };
 
@@ -292,7 +295,32 @@ __device__ __forceinline__ void store_chunk(const ContractionArgs& p, long long 
                 v[j + 3] = __fadd_rn(v[j + 3], b4.w);
             }
         }
-        if (!p.y_is_bf16) {
+        if (p.y_is_i8) {
+            // the next layer's INT8 activations: ReLU, one multiply by fl(1 / out_scale), round half to even, clip
+            int8_t* dst = reinterpret_cast<int8_t*>(p.y) + row * p.ldy + col0;
+            uint32_t w[8];
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+                uint32_t word = 0;
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    float t = p.relu ? fmaxf(v[j + b], 0.0f) : v[j + b];
+                    int q = __float2int_rn(__fmul_rn(t, p.inv_out_scale));
+                    q = max(-128, min(127, q));
+                    word |= (uint32_t)(q & 0xff) << (8 * b);
+                }
+                w[j >> 2] = word;
+            }
+            const bool vec_i8 = ((p.ldy & 15) == 0) && ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
+            if (full_chunk && vec_i8) {
+                *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+                *reinterpret_cast<uint4*>(dst + 16) = make_uint4(w[4], w[5], w[6], w[7]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                    if (col0 + j < p.N) dst[j] = (int8_t)((w[j >> 2] >> (8 * (j & 3))) & 0xffu);
+            }
+        } else if (!p.y_is_bf16) {
             float* dst = reinterpret_cast<float*>(p.y) + row * p.ldy + col0;
             if (full_chunk && vec_f32) {
 #pragma unroll
@@ -384,7 +412,7 @@ __device__ __forceinline__ void store_chunk_warp(const ContractionArgs& p, int r
                                                  const CUtensorMap* tmY, const CUtensorMap* tmAcc, const OutCoords& oc) {
     const bool full_chunk = col0 + 32 <= p.N;
     const bool acc_fast = p.acc_out == nullptr || p.acc_tma || (full_chunk && vec_acc);
-    const bool y_fast = p.y == nullptr || p.y_tma || (full_chunk && (p.y_is_bf16 ? vec_bf16 : vec_f32));
+    const bool y_fast = p.y == nullptr || (!p.y_is_i8 && (p.y_tma || (full_chunk && (p.y_is_bf16 ? vec_bf16 : vec_f32))));
     if (!acc_fast || !y_fast) {                        // ragged or unaligned: the plain per-row path
         if (row_ok) store_chunk(p, row, col0, r, sc, bs, vec_acc, vec_f32, vec_bf16);
         return;
@@ -788,11 +816,19 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     }
 }
 
+// Output type used inside the library for the requantised INT8 result, and its parameters.
+constexpr int kOutI8 = 2;
+struct OutQuant {
+    float out_scale;
+    int relu;
+};
+
 // Host launcher (defined with the GEMM entry points).  The A operand is reached through tmA: a plain 2-D map
 // of an [M, K] matrix (kModeGemm, geom == nullptr) or a 4-D map of NHWC activations (convolution modes).
 int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int m_tiles, int k_blocks,
                     const void* Bmat, int64_t ldb, bool part, int n_bits, int h_bits,
                     const float* w_scale, float act_scale, const float* bias, int64_t M, int64_t N, int64_t K,
-                    int32_t* acc_out, int64_t ld_acc, void* Y, int64_t ldy, int y_dtype, cudaStream_t stream);
+                    int32_t* acc_out, int64_t ld_acc, void* Y, int64_t ldy, int y_dtype, cudaStream_t stream,
+                    const OutQuant* oq = nullptr);
 
 }  // namespace nq

@@ -217,12 +217,14 @@ int64_t nq_conv_workspace_bytes(const nq_conv_desc* d) {
     return (int64_t)d->B * Ho * Wo * ((K + 15) / 16 * 16);
 }
 
-int nq_conv_implicit_gemm(const int8_t* X, const void* Wt, int64_t ldw, int part_bit, int n_bits, int h_bits,
-                          const nq_conv_desc* d, const float* w_scale, float act_scale, const float* bias,
-                          int32_t* acc_out, void* Y, int y_dtype, void* workspace, int64_t workspace_bytes, void* stream_) {
+static int conv_common(const int8_t* X, const void* Wt, int64_t ldw, int part_bit, int n_bits, int h_bits,
+                       const nq_conv_desc* d, const float* w_scale, float act_scale, const float* bias,
+                       int32_t* acc_out, void* Y, int y_dtype, void* workspace, int64_t workspace_bytes, void* stream_,
+                       const nq::OutQuant* oq) {
     using namespace nq;
     if (!desc_ok(d)) return NQ_ERR_INVALID_ARG;
-    if (y_dtype != NQ_F32 && y_dtype != NQ_BF16) return NQ_ERR_INVALID_ARG;
+    if (y_dtype != NQ_F32 && y_dtype != NQ_BF16 && !(y_dtype == kOutI8 && oq)) return NQ_ERR_INVALID_ARG;
+    if (oq && !(oq->out_scale > 0.0f)) return NQ_ERR_INVALID_ARG;
     if (part_bit && (n_bits < 2 || n_bits > 8 || h_bits < 1 || h_bits >= n_bits)) return NQ_ERR_UNSUPPORTED;
     if (!X || !Wt || (!acc_out && !Y) || (Y && !w_scale)) return NQ_ERR_INVALID_ARG;
     const int Ho = out_dim(d->H, d->R, d->stride, d->pad), Wo = out_dim(d->W, d->S, d->stride, d->pad);
@@ -253,7 +255,7 @@ int nq_conv_implicit_gemm(const int8_t* X, const void* Wt, int64_t ldw, int part
         if (st != NQ_OK) return st;
         return run_contraction(tmA, kModeGemm, nullptr, (int)((M + kBM - 1) / kBM), (int)((K + kBK - 1) / kBK), Wt, ldw,
                                part_bit != 0, n_bits, h_bits, w_scale, act_scale, bias, M, N, K, acc_out, N, Y, N, y_dtype,
-                               stream);
+                               stream, oq);
     }
 
     const int8_t* x_nhwc = X;
@@ -286,7 +288,24 @@ int nq_conv_implicit_gemm(const int8_t* X, const void* Wt, int64_t ldw, int part
     }
     if (st != NQ_OK) return st;
     return run_contraction(tmA, mode, &g, m_tiles, k_blocks, Wt, ldw, part_bit != 0, n_bits, h_bits, w_scale, act_scale,
-                           bias, M, N, K, acc_out, N, Y, N, y_dtype, stream);
+                           bias, M, N, K, acc_out, N, Y, N, y_dtype, stream, oq);
+}
+
+int nq_conv_implicit_gemm(const int8_t* X, const void* Wt, int64_t ldw, int part_bit, int n_bits, int h_bits,
+                          const nq_conv_desc* d, const float* w_scale, float act_scale, const float* bias,
+                          int32_t* acc_out, void* Y, int y_dtype, void* workspace, int64_t workspace_bytes, void* stream) {
+    if (y_dtype != NQ_F32 && y_dtype != NQ_BF16) return NQ_ERR_INVALID_ARG;
+    return conv_common(X, Wt, ldw, part_bit, n_bits, h_bits, d, w_scale, act_scale, bias, acc_out, Y, y_dtype, workspace,
+                       workspace_bytes, stream, nullptr);
+}
+
+int nq_conv_implicit_gemm_q8(const int8_t* X, const void* Wt, int64_t ldw, int part_bit, int n_bits, int h_bits,
+                             const nq_conv_desc* d, const float* w_scale, float act_scale, const float* bias,
+                             float out_scale, int relu, int8_t* Yq, void* workspace, int64_t workspace_bytes, void* stream) {
+    const nq::OutQuant oq{out_scale, relu};
+    if (!Yq) return NQ_ERR_INVALID_ARG;
+    return conv_common(X, Wt, ldw, part_bit, n_bits, h_bits, d, w_scale, act_scale, bias, nullptr, Yq, nq::kOutI8, workspace,
+                       workspace_bytes, stream, &oq);
 }
 
 int nq_conv_implicit_gemm_static(const int8_t* X, const void* Wt, int64_t ldw, int part_bit, int n_bits, int h_bits,

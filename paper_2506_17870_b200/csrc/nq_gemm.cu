@@ -201,7 +201,8 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int m_tiles, int k_blocks,
                     const void* Bmat, int64_t ldb, bool part, int n_bits, int h_bits,
                     const float* w_scale, float act_scale, const float* bias, int64_t M, int64_t N, int64_t K,
-                    int32_t* acc_out, int64_t ld_acc, void* Y, int64_t ldy, int y_dtype, cudaStream_t stream) {
+                    int32_t* acc_out, int64_t ld_acc, void* Y, int64_t ldy, int y_dtype, cudaStream_t stream,
+                    const OutQuant* oq) {
     // Tile shape: the widest tile reuses operands best, but a small problem must first of all fill the
     // machine.  Estimate, for each candidate, (waves of tiles over the SMs) x (stages per tile) x (cycles per
     // stage, measured orders of magnitude: narrow tiles are load-bound, the wide single-CTA tile is
@@ -237,11 +238,14 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
     a.div_last = make_fastdiv((uint32_t)((a.m_tiles % kGroupM) ? (a.m_tiles % kGroupM) : 1));
     a.w_scale = w_scale; a.bias = bias; a.act_scale = act_scale;
     a.acc_out = acc_out; a.ld_acc = ld_acc; a.y = Y; a.ldy = ldy; a.y_is_bf16 = (y_dtype == NQ_BF16);
+    a.y_is_i8 = (y_dtype == kOutI8 && oq) ? 1 : 0;
+    a.relu = oq ? oq->relu : 0;
+    a.inv_out_scale = oq ? 1.0f / oq->out_scale : 1.0f;
     a.status = status_word();
     if (!a.status) return NQ_ERR_CUDA;
     OutMaps om;
     om.y = tmA; om.acc = tmA;
-    a.y_tma = make_out_map(&om.y, Y, y_dtype == NQ_BF16 ? 2 : 4, M, N, ldy, geom) ? 1 : 0;
+    a.y_tma = (!a.y_is_i8 && make_out_map(&om.y, Y, y_dtype == NQ_BF16 ? 2 : 4, M, N, ldy, geom)) ? 1 : 0;
     a.acc_tma = make_out_map(&om.acc, acc_out, 4, M, N, ld_acc, geom) ? 1 : 0;
     CUtensorMap tmB;
     bool direct = false;
@@ -290,9 +294,11 @@ namespace {
 
 int gemm_common(const int8_t* X, int64_t ldx, const void* Bmat, int64_t ldb, bool part, int n_bits, int h_bits,
                 const float* w_scale, float act_scale, const float* bias, int64_t M, int64_t N, int64_t K,
-                int32_t* acc_out, int64_t ld_acc, void* Y, int64_t ldy, int y_dtype, void* stream) {
+                int32_t* acc_out, int64_t ld_acc, void* Y, int64_t ldy, int y_dtype, void* stream,
+                const OutQuant* oq = nullptr) {
     if (M < 0 || N < 0 || K < 0) return NQ_ERR_INVALID_ARG;
-    if (y_dtype != NQ_F32 && y_dtype != NQ_BF16) return NQ_ERR_INVALID_ARG;
+    if (y_dtype != NQ_F32 && y_dtype != NQ_BF16 && !(y_dtype == kOutI8 && oq)) return NQ_ERR_INVALID_ARG;
+    if (oq && !(oq->out_scale > 0.0f)) return NQ_ERR_INVALID_ARG;
     if (part && (n_bits < 2 || n_bits > 8 || h_bits < 1 || h_bits >= n_bits)) return NQ_ERR_UNSUPPORTED;
     if (K >= (1 << 17) || M > (1ll << 30) || N > (1ll << 30)) return NQ_ERR_UNSUPPORTED;
     if (M == 0 || N == 0) return NQ_OK;
@@ -302,14 +308,14 @@ int gemm_common(const int8_t* X, int64_t ldx, const void* Bmat, int64_t ldb, boo
     if (K == 0) return NQ_ERR_UNSUPPORTED;
     if (!X || !Bmat || ldx < K || (!part && ldb < K)) return NQ_ERR_INVALID_ARG;
     if (!aligned16(X) || (ldx & 15) || !aligned16(Bmat) || (!part && (ldb & 15))) return NQ_ERR_ALIGNMENT;
-    if ((acc_out && (reinterpret_cast<uintptr_t>(acc_out) & 3)) || (Y && (reinterpret_cast<uintptr_t>(Y) & 1)))
+    if ((acc_out && (reinterpret_cast<uintptr_t>(acc_out) & 3)) || (Y && y_dtype != kOutI8 && (reinterpret_cast<uintptr_t>(Y) & 1)))
         return NQ_ERR_ALIGNMENT;
     CUtensorMap tmA;
     int st = encode_tensor_map_2d(&tmA, X, (uint64_t)K, (uint64_t)M, (uint64_t)ldx, kBK, kBM, 128);
     if (st != NQ_OK) return st;
     return run_contraction(tmA, kModeGemm, nullptr, (int)((M + kBM - 1) / kBM), (int)((K + kBK - 1) / kBK), Bmat, ldb,
                            part, n_bits, h_bits, w_scale, act_scale, bias, M, N, K, acc_out, ld_acc, Y, ldy, y_dtype,
-                           (cudaStream_t)stream);
+                           (cudaStream_t)stream, oq);
 }
 
 }  // namespace
@@ -322,6 +328,24 @@ int nq_gemm_full(const int8_t* X, int64_t ldx, const int8_t* W, int64_t ldw, con
                  int64_t ldy, int y_dtype, void* stream) {
     return nq::gemm_common(X, ldx, W, ldw, false, 8, 0, w_scale, act_scale, bias, M, N, K, acc_out, ld_acc, Y, ldy,
                            y_dtype, stream);
+}
+
+int nq_gemm_full_q8(const int8_t* X, int64_t ldx, const int8_t* W, int64_t ldw, const float* w_scale, float act_scale,
+                    const float* bias, float out_scale, int relu, int64_t M, int64_t N, int64_t K, int8_t* Yq,
+                    int64_t ldyq, void* stream) {
+    const nq::OutQuant oq{out_scale, relu};
+    if (!Yq) return NQ_ERR_INVALID_ARG;
+    return nq::gemm_common(X, ldx, W, ldw, false, 8, 0, w_scale, act_scale, bias, M, N, K, nullptr, 0, Yq, ldyq, nq::kOutI8,
+                           stream, &oq);
+}
+
+int nq_gemm_part_q8(const int8_t* X, int64_t ldx, const void* packed_high, int n_bits, int h_bits, const float* w_scale,
+                    float act_scale, const float* bias, float out_scale, int relu, int64_t M, int64_t N, int64_t K,
+                    int8_t* Yq, int64_t ldyq, void* stream) {
+    const nq::OutQuant oq{out_scale, relu};
+    if (!Yq) return NQ_ERR_INVALID_ARG;
+    return nq::gemm_common(X, ldx, packed_high, 0, true, n_bits, h_bits, w_scale, act_scale, bias, M, N, K, nullptr, 0, Yq,
+                           ldyq, nq::kOutI8, stream, &oq);
 }
 
 int nq_gemm_part(const int8_t* X, int64_t ldx, const void* packed_high, int n_bits, int h_bits, const float* w_scale,
