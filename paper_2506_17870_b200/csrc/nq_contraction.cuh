@@ -253,6 +253,24 @@ __device__ __forceinline__ TileOrigin conv_tile_origin(const ConvGeom& g, int mt
     return o;
 }
 
+// Four dequantised values -> four INT8 activations in one word (byte i = value i): one multiply by fl(1 / out_scale),
+// round half to even, clip.  The conversion saturates to int32, the packing instruction to INT8; with ReLU the
+// packing saturates to [0, 255] instead and a per-byte minimum brings that to [0, 127] (a negative value rounds to
+// a non-positive integer, so clipping at zero after the rounding equals ReLU before it).
+__device__ __forceinline__ uint32_t requant4(float v0, float v1, float v2, float v3, float inv, int relu) {
+    const int q0 = __float2int_rn(__fmul_rn(v0, inv)), q1 = __float2int_rn(__fmul_rn(v1, inv));
+    const int q2 = __float2int_rn(__fmul_rn(v2, inv)), q3 = __float2int_rn(__fmul_rn(v3, inv));
+    uint32_t hi, out;
+    if (relu) {
+        asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(q3), "r"(q2), "r"(0u));
+        asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(out) : "r"(q1), "r"(q0), "r"(hi));
+        return __vminu4(out, 0x7f7f7f7fu);
+    }
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(q3), "r"(q2), "r"(0u));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(out) : "r"(q1), "r"(q0), "r"(hi));
+    return out;
+}
+
 // Epilogue of one thread for 32 consecutive columns of its output row: optional int32 copy (with the
 // part-bit shift), dequantisation in the stated rounding order, fp32 or bf16 store; vector stores when
 // the chunk is whole and the pointers and pitches allow.
@@ -300,17 +318,7 @@ __device__ __forceinline__ void store_chunk(const ContractionArgs& p, long long 
             int8_t* dst = reinterpret_cast<int8_t*>(p.y) + row * p.ldy + col0;
             uint32_t w[8];
 #pragma unroll
-            for (int j = 0; j < 32; j += 4) {
-                uint32_t word = 0;
-#pragma unroll
-                for (int b = 0; b < 4; ++b) {
-                    float t = p.relu ? fmaxf(v[j + b], 0.0f) : v[j + b];
-                    int q = __float2int_rn(__fmul_rn(t, p.inv_out_scale));
-                    q = max(-128, min(127, q));
-                    word |= (uint32_t)(q & 0xff) << (8 * b);
-                }
-                w[j >> 2] = word;
-            }
+            for (int j = 0; j < 32; j += 4) w[j >> 2] = requant4(v[j], v[j + 1], v[j + 2], v[j + 3], p.inv_out_scale, p.relu);
             const bool vec_i8 = ((p.ldy & 15) == 0) && ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
             if (full_chunk && vec_i8) {
                 *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -405,6 +413,24 @@ __device__ __forceinline__ void store_rows64_tma(uint8_t* stage, int lane, const
     }
 }
 
+// The same for 32-byte rows (INT8 output): a 32 x 32-byte block in the 32-byte swizzle.
+__device__ __forceinline__ void store_rows32_tma(uint8_t* stage, int lane, const uint4 (&q)[2], const CUtensorMap* map,
+                                                 int x_byte, const OutCoords& oc) {
+    using namespace sm100;
+    if (lane == 0) bulk_wait_read_all();
+    __syncwarp();
+    uint8_t* mine = stage + lane * 32;
+    const int sw = (lane >> 2) & 1;
+    *reinterpret_cast<uint4*>(mine + ((0 ^ sw) << 4)) = q[0];
+    *reinterpret_cast<uint4*>(mine + ((1 ^ sw) << 4)) = q[1];
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+        tma_store_4d(map, smem_u32(stage), x_byte, oc.c1, oc.c2, oc.c3);
+        bulk_commit_group();
+    }
+}
+
 // The epilogue of one warp for 32 consecutive columns: same arithmetic as store_chunk, coalesced stores.
 __device__ __forceinline__ void store_chunk_warp(const ContractionArgs& p, int row, bool row_ok, int col0,
                                                  const uint32_t (&r)[32], const float* sc, const float* bs,
@@ -412,7 +438,7 @@ __device__ __forceinline__ void store_chunk_warp(const ContractionArgs& p, int r
                                                  const CUtensorMap* tmY, const CUtensorMap* tmAcc, const OutCoords& oc) {
     const bool full_chunk = col0 + 32 <= p.N;
     const bool acc_fast = p.acc_out == nullptr || p.acc_tma || (full_chunk && vec_acc);
-    const bool y_fast = p.y == nullptr || (!p.y_is_i8 && (p.y_tma || (full_chunk && (p.y_is_bf16 ? vec_bf16 : vec_f32))));
+    const bool y_fast = p.y == nullptr || p.y_tma || (!p.y_is_i8 && full_chunk && (p.y_is_bf16 ? vec_bf16 : vec_f32));
     if (!acc_fast || !y_fast) {                        // ragged or unaligned: the plain per-row path
         if (row_ok) store_chunk(p, row, col0, r, sc, bs, vec_acc, vec_f32, vec_bf16);
         return;
@@ -452,7 +478,14 @@ __device__ __forceinline__ void store_chunk_warp(const ContractionArgs& p, int r
                 v[j + 3] = __fadd_rn(v[j + 3], b4.w);
             }
         }
-        if (!p.y_is_bf16) {
+        if (p.y_is_i8) {
+            // the next layer's INT8 activations: ReLU, one multiply by fl(1 / out_scale), round half to even, clip
+            uint32_t w8[8];
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) w8[j >> 2] = requant4(v[j], v[j + 1], v[j + 2], v[j + 3], p.inv_out_scale, p.relu);
+            const uint4 q2[2] = {make_uint4(w8[0], w8[1], w8[2], w8[3]), make_uint4(w8[4], w8[5], w8[6], w8[7])};
+            store_rows32_tma(stage, lane, q2, tmY, col0, oc);
+        } else if (!p.y_is_bf16) {
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
 #pragma unroll

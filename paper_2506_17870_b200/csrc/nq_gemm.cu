@@ -62,15 +62,16 @@ int encode_tensor_map_nhwc(CUtensorMap* map, const void* base, uint64_t C, uint6
 }
 
 int encode_tensor_map_out(CUtensorMap* map, const void* base, uint64_t row_bytes, uint64_t pitch_bytes, uint64_t d1,
-                          uint64_t d2, uint64_t d3, uint32_t b1, uint32_t b2, uint32_t b3) {
+                          uint64_t d2, uint64_t d3, uint32_t b1, uint32_t b2, uint32_t b3, uint32_t box_bytes) {
     EncodeFn fn = encode_fn();
     if (!fn) return NQ_ERR_CUDA;
     cuuint64_t dims[4] = {row_bytes, d1, d2, d3};
     cuuint64_t strides[3] = {pitch_bytes, pitch_bytes * d1, pitch_bytes * d1 * d2};
-    cuuint32_t box[4] = {64, b1, b2, b3};
+    cuuint32_t box[4] = {box_bytes, b1, b2, b3};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, box_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_64B,
+                    CU_TENSOR_MAP_L2_PROMOTION_NONE,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? NQ_OK : NQ_ERR_CUDA;
 }
@@ -166,12 +167,14 @@ bool make_out_map(CUtensorMap* map, const void* base, int esize, int64_t M, int6
     if (!base || !tile_stores_enabled()) return false;
     const uint64_t pitch = (uint64_t)ld * esize, row_bytes = (uint64_t)N * esize;
     if ((reinterpret_cast<uintptr_t>(base) & 15) || (pitch & 15) || pitch >= (1ull << 40)) return false;
-    if (!g) return encode_tensor_map_out(map, base, row_bytes, pitch, (uint64_t)M, 1, 1, 32, 1, 1) == NQ_OK;
+    const uint32_t box_bytes = esize == 1 ? 32 : 64;      // 32 columns of the output
+    if (!g) return encode_tensor_map_out(map, base, row_bytes, pitch, (uint64_t)M, 1, 1, 32, 1, 1, box_bytes) == NQ_OK;
     const uint32_t tw = 1u << g->tw_log2, th = 1u << g->th_log2;
     const uint32_t bw = tw < 32 ? tw : 32;
     const uint32_t bh = (32 / bw) < th ? (32 / bw) : th;
     const uint32_t bb = 32 / (bw * bh);
-    return encode_tensor_map_out(map, base, row_bytes, pitch, (uint64_t)g->Wo, (uint64_t)g->Ho, (uint64_t)g->B, bw, bh, bb) == NQ_OK;
+    return encode_tensor_map_out(map, base, row_bytes, pitch, (uint64_t)g->Wo, (uint64_t)g->Ho, (uint64_t)g->B, bw, bh, bb,
+                                 box_bytes) == NQ_OK;
 }
 
 // NQ_PACKED_RING=1 in the environment keeps every part-bit pair launch on the TMA-fed ring of packed tiles
@@ -245,7 +248,7 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
     if (!a.status) return NQ_ERR_CUDA;
     OutMaps om;
     om.y = tmA; om.acc = tmA;
-    a.y_tma = (!a.y_is_i8 && make_out_map(&om.y, Y, y_dtype == NQ_BF16 ? 2 : 4, M, N, ldy, geom)) ? 1 : 0;
+    a.y_tma = make_out_map(&om.y, Y, a.y_is_i8 ? 1 : (y_dtype == NQ_BF16 ? 2 : 4), M, N, ldy, geom) ? 1 : 0;
     a.acc_tma = make_out_map(&om.acc, acc_out, 4, M, N, ld_acc, geom) ? 1 : 0;
     CUtensorMap tmB;
     bool direct = false;

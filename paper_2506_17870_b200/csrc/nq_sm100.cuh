@@ -311,8 +311,8 @@ int encode_tensor_map_2d(CUtensorMap* map, const void* base, uint64_t inner, uin
 int encode_tensor_map_nhwc(CUtensorMap* map, const void* base, uint64_t C, uint64_t W, uint64_t H, uint64_t B,
                            uint32_t box_c, uint32_t tw, uint32_t th, uint32_t tb, uint32_t stride, int swizzle_bytes);
 // Output matrix as a 4-D byte tensor (row bytes, d1, d2, d3) for the epilogue's tile stores: boxes of 64 bytes x
-// b1 x b2 x b3 rows (32 rows in all) in the 64-byte swizzle.  A plain [M, N] matrix is (N * esize, M, 1, 1).
+// b1 x b2 x b3 rows (32 rows in all) in the 64-byte swizzle (32-byte rows and swizzle for INT8 output).  A plain [M, N] matrix is (N * esize, M, 1, 1).
 int encode_tensor_map_out(CUtensorMap* map, const void* base, uint64_t row_bytes, uint64_t pitch_bytes, uint64_t d1,
-                          uint64_t d2, uint64_t d3, uint32_t b1, uint32_t b2, uint32_t b3);
+                          uint64_t d2, uint64_t d3, uint32_t b1, uint32_t b2, uint32_t b3, uint32_t box_bytes = 64);
 
 }  // namespace nq
