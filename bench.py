@@ -536,6 +536,35 @@ def _model_rows(nq, torch, wl, dev, conv_batch):
         res["part_bit" if part else "full_bit"] = {"ms": round(ms, 3), "tops": round(ops / (ms * 1e-3) / 1e12, 1)}
     res.update({"layers": len(layers), "batch": conv_batch, "weights": sum(L.weights for L in layers),
                 "tera_ops_per_pass": round(ops / 1e12, 3)})
+    # the same stack in chained form: NHWC int8 activations in, the next layer's INT8 activations out (requantising
+    # epilogue with ReLU), no layout pre-pass; every layer still runs on its own input
+    yq = torch.empty(y_elems, dtype=torch.int8, device=dev)
+    for cs, L in zip(prepared, layers):
+        key = ("nhwc", L.Cin, L.H, L.W)
+        if key not in xs:
+            xs[key] = cs["x"].permute(0, 2, 3, 1).contiguous()
+        cs["x_nhwc"] = xs[key]
+        cs["desc_nhwc"] = nq.nq_conv_desc(conv_batch, L.Cin, L.H, L.W, L.Cout, L.R, L.S, L.stride, L.pad, 0)
+        cs["yq"] = yq[:conv_batch * L.Ho * L.Wo * L.Cout].view(conv_batch, L.Ho, L.Wo, L.Cout)
+    for part in (False, True):
+        per_layer = []
+        for rep in range(4):
+            evs = []
+            for cs in prepared:
+                a = torch.cuda.Event(enable_timing=True)
+                b = torch.cuda.Event(enable_timing=True)
+                a.record()
+                nq.nq_conv_implicit_gemm_q8(cs["x_nhwc"], cs["hi"] if part else cs["w"], cs["desc_nhwc"], cs["ws"], cs["act"],
+                                            0.5, relu=True, part_bit=part, n_bits=N_BITS, h_bits=CONV_H,
+                                            workspace=cs["work"], y_out=cs["yq"])
+                b.record()
+                evs.append((a, b))
+            torch.cuda.synchronize()
+            if rep:
+                per_layer.append([a.elapsed_time(b) for a, b in evs])
+        ms = float(np.sum(np.median(np.array(per_layer), axis=0)))
+        res["chained_int8_out_" + ("part_bit" if part else "full_bit")] = {"ms": round(ms, 3), "tops": round(ops / (ms * 1e-3) / 1e12, 1)}
+    del yq
     out["resnet101_stack_int8_6"] = res
     nq.nq_device_status()
     del prepared, xs, ybuf, work

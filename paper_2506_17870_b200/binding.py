@@ -341,7 +341,8 @@ def nq_gemm_part_q8(X: torch.Tensor, packed_high: torch.Tensor, N: int, n_bits: 
 
 def nq_conv_implicit_gemm_q8(X: torch.Tensor, Wt: torch.Tensor, desc: nq_conv_desc, w_scale: torch.Tensor, act_scale: float,
                              out_scale: float, relu: bool = True, part_bit: bool = False, n_bits: int = 8, h_bits: int = 6,
-                             bias: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+                             bias: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                             y_out: Optional[torch.Tensor] = None) -> torch.Tensor:
     """Convolution whose NHWC output is the next layer's INT8 activations."""
     Ho = (desc.H + 2 * desc.pad - desc.R) // desc.stride + 1
     Wo = (desc.W + 2 * desc.pad - desc.S) // desc.stride + 1
@@ -349,7 +350,7 @@ def nq_conv_implicit_gemm_q8(X: torch.Tensor, Wt: torch.Tensor, desc: nq_conv_de
     if workspace is None:
         workspace = torch.empty(max(need, 0) + 2048, dtype=torch.uint8, device=X.device)
     off = (-workspace.data_ptr()) % 1024
-    y = torch.empty((desc.B, Ho, Wo, desc.Cout), dtype=torch.int8, device=X.device)
+    y = y_out if y_out is not None else torch.empty((desc.B, Ho, Wo, desc.Cout), dtype=torch.int8, device=X.device)
     ldw = _ld(Wt) if not part_bit else 0
     _check(lib().nq_conv_implicit_gemm_q8(_ptr(X), _ptr(Wt), _i64(ldw), int(bool(part_bit)), n_bits, h_bits,
                                           ctypes.byref(desc), _ptr(w_scale), ctypes.c_float(act_scale), _ptr(bias),
