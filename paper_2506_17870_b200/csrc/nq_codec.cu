@@ -423,6 +423,46 @@ __global__ void __launch_bounds__(256, 4) codec_batched_kernel(const BatchEntry*
     }
 }
 
+// The paper's packed-bit words (64 // BITS fields per 64-bit word) -> sliced layout.  One thread per 32-element
+// unit: it walks the words that hold its fields, drops each field into the top bits of its byte lane of the
+// eight top-aligned words, and lets store_unit_top cut the slices -- the same last step as every codec kernel.
+template <int BITS>
+__global__ void __launch_bounds__(256) word64_to_sliced_kernel(const uint64_t* __restrict__ words, int64_t rows,
+                                                               int64_t cols, uint8_t* __restrict__ packed) {
+    constexpr int PER = 64 / BITS;
+    constexpr uint32_t MASK = (1u << BITS) - 1u;
+    const int64_t units_per_row = ((cols + 127) >> 7) << 2;
+    const int64_t row_words = (cols + PER - 1) / PER;
+    const int64_t total = rows * units_per_row;
+    for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < total; u += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = u / units_per_row, ur = u - row * units_per_row;
+        const int64_t c0 = ur * 32;
+        const uint64_t* wrow = words + row * row_words;
+        int64_t wi = c0 / PER;
+        int fi = (int)(c0 - wi * PER);
+        uint64_t w = (c0 < cols) ? __ldg(wrow + wi) >> (fi * BITS) : 0ull;
+        uint32_t T[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            uint32_t t = 0;
+#pragma unroll
+            for (int lane = 0; lane < 4; ++lane) {
+                const int j = q * 4 + lane;
+                const uint32_t f = (c0 + j < cols) ? ((uint32_t)w & MASK) : 0u;
+                t |= f << (8 * lane + 8 - BITS);
+                w >>= BITS;
+                if (++fi == PER) {
+                    fi = 0;
+                    ++wi;
+                    w = (c0 + j + 1 < cols) ? __ldg(wrow + wi) : 0ull;
+                }
+            }
+            T[q] = t;
+        }
+        store_unit_top(packed + (row * (units_per_row >> 2) + (ur >> 2)) * 16 * BITS, (int)(ur & 3), BITS, T);
+    }
+}
+
 inline int launch_blocks(int64_t total_units) {
     int64_t need = (total_units + 255) / 256;
     int64_t cap = (int64_t)nq::sm_count() * 8 * 4;
@@ -488,6 +528,24 @@ int run_single(TensorView t, int n, int h, int comp, int bits, void* stream) {
 }
 
 }  // namespace
+
+namespace nq {
+int word64_to_sliced_launch(const uint64_t* words, int bits, int64_t rows, int64_t cols, uint8_t* packed, cudaStream_t s) {
+    const int64_t units = rows * (((cols + 127) >> 7) << 2);
+    const int blocks = launch_blocks(units);
+    switch (bits) {
+        case 1: word64_to_sliced_kernel<1><<<blocks, 256, 0, s>>>(words, rows, cols, packed); break;
+        case 2: word64_to_sliced_kernel<2><<<blocks, 256, 0, s>>>(words, rows, cols, packed); break;
+        case 3: word64_to_sliced_kernel<3><<<blocks, 256, 0, s>>>(words, rows, cols, packed); break;
+        case 4: word64_to_sliced_kernel<4><<<blocks, 256, 0, s>>>(words, rows, cols, packed); break;
+        case 5: word64_to_sliced_kernel<5><<<blocks, 256, 0, s>>>(words, rows, cols, packed); break;
+        case 6: word64_to_sliced_kernel<6><<<blocks, 256, 0, s>>>(words, rows, cols, packed); break;
+        case 7: word64_to_sliced_kernel<7><<<blocks, 256, 0, s>>>(words, rows, cols, packed); break;
+        default: word64_to_sliced_kernel<8><<<blocks, 256, 0, s>>>(words, rows, cols, packed); break;
+    }
+    return cudaGetLastError() == cudaSuccess ? NQ_OK : NQ_ERR_CUDA;
+}
+}  // namespace nq
 
 extern "C" {
 

@@ -12,5 +12,8 @@ int sm_count();
 // Defined in nq_runtime.cu; kernels get its address through status_word().
 unsigned int* status_word();
 
+// The paper's 64-bit packed words -> sliced layout (kernel beside the codec, whose slice cutter it uses).
+int word64_to_sliced_launch(const uint64_t* words, int bits, int64_t rows, int64_t cols, uint8_t* packed, cudaStream_t s);
+
 }  // namespace nq
 

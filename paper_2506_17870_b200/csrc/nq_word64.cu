@@ -4,8 +4,8 @@
 // 64 // k fields each, field j at bits [j*k, j*k + k), the unused top bits zero (twenty-one 3-bit or twelve
 // 5-bit weights per word).  That is the format a model arrives in; the kernels of this library work on the
 // sliced layout of nq.h.  Both directions are plain element-wise moves of k-bit two's-complement fields:
-//   word64 -> sliced   one thread per 32-element unit: walks the words that hold its fields, then lays the
-//                      unit's slices down word by word
+//   word64 -> sliced   one thread per 32-element unit, in nq_codec.cu beside the slice cutter it shares with
+//                      the codec kernels
 //   sliced -> word64   one thread per output word: gathers its 64 // k fields out of the slices
 // They are conversion utilities (run once per model), written for clarity; the hot codec is nq_codec.cu.
 #include <cuda_runtime.h>
@@ -24,59 +24,6 @@ __device__ __forceinline__ void slice_place(int s, int e, int& byte_off, int& sh
     const int word = q / per_byte, sub = q - word * per_byte;
     byte_off = ((unit * s + word) << 2) + lane;
     shift = 8 - s * sub - s;
-}
-
-template <int BITS>
-__global__ void __launch_bounds__(256) word64_to_sliced_kernel(const uint64_t* __restrict__ words, int64_t rows,
-                                                               int64_t cols, uint8_t* __restrict__ packed) {
-    constexpr int PER = 64 / BITS;
-    constexpr uint64_t MASK = (1ull << BITS) - 1ull;
-    const int64_t units_per_row = ((cols + 127) >> 7) << 2;
-    const int64_t row_words = (cols + PER - 1) / PER;
-    const int64_t total = rows * units_per_row;
-    for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < total; u += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t row = u / units_per_row, ur = u - row * units_per_row;
-        const int64_t c0 = ur * 32;
-        const uint64_t* wrow = words + row * row_words;
-        // the unit's 32 fields, read in order: the word index and the position inside the word advance together
-        uint32_t f[32];
-        int64_t wi = c0 / PER;
-        int fi = (int)(c0 - wi * PER);
-        uint64_t w = (c0 < cols) ? wrow[wi] : 0ull;
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            f[j] = (c0 + j < cols) ? (uint32_t)((w >> (fi * BITS)) & MASK) : 0u;
-            if (++fi == PER) {
-                fi = 0;
-                ++wi;
-                w = (c0 + j + 1 < cols) ? wrow[wi] : 0ull;
-            }
-        }
-        uint8_t* group = packed + (row * (units_per_row >> 2) + (ur >> 2)) * 16 * BITS;
-        const int unit = (int)(ur & 3);
-        int used = 0, slice_base = 0;
-#pragma unroll
-        for (int s = 8; s >= 1; s >>= 1) {
-            if (!(BITS & s)) continue;
-            const int per_byte = 8 / s;
-#pragma unroll
-            for (int wq = 0; wq < s; ++wq) {
-                uint32_t out = 0;
-#pragma unroll
-                for (int sub = 0; sub < per_byte; ++sub) {
-                    const int q = wq * per_byte + sub;
-#pragma unroll
-                    for (int lane = 0; lane < 4; ++lane) {
-                        const uint32_t part = (f[q * 4 + lane] >> (BITS - used - s)) & ((1u << s) - 1u);
-                        out |= part << ((8 - s * sub - s) + 8 * lane);
-                    }
-                }
-                *reinterpret_cast<uint32_t*>(group + slice_base + ((unit * s + wq) << 2)) = out;
-            }
-            slice_base += 16 * s;
-            used += s;
-        }
-    }
 }
 
 template <int BITS>
@@ -118,16 +65,10 @@ inline int blocks_for(int64_t threads) {
 }
 
 template <int BITS>
-int launch_bits(bool to_sliced, const void* src, int64_t rows, int64_t cols, void* dst, cudaStream_t s) {
-    if (to_sliced) {
-        const int64_t units = rows * (((cols + 127) >> 7) << 2);
-        word64_to_sliced_kernel<BITS><<<blocks_for(units), 256, 0, s>>>(static_cast<const uint64_t*>(src), rows, cols,
-                                                                       static_cast<uint8_t*>(dst));
-    } else {
-        const int64_t n = rows * ((cols + 64 / BITS - 1) / (64 / BITS));
-        sliced_to_word64_kernel<BITS><<<blocks_for(n), 256, 0, s>>>(static_cast<const uint8_t*>(src), rows, cols,
-                                                                    static_cast<uint64_t*>(dst));
-    }
+int launch_from_sliced(const void* src, int64_t rows, int64_t cols, void* dst, cudaStream_t s) {
+    const int64_t n = rows * ((cols + 64 / BITS - 1) / (64 / BITS));
+    sliced_to_word64_kernel<BITS><<<blocks_for(n), 256, 0, s>>>(static_cast<const uint8_t*>(src), rows, cols,
+                                                                static_cast<uint64_t*>(dst));
     return cudaGetLastError() == cudaSuccess ? NQ_OK : NQ_ERR_CUDA;
 }
 
@@ -140,15 +81,17 @@ int convert(bool to_sliced, const void* src, int bits, int64_t rows, int64_t col
     const void* w64 = to_sliced ? src : dst;
     if ((reinterpret_cast<uintptr_t>(sliced) & 15) || (reinterpret_cast<uintptr_t>(w64) & 7)) return NQ_ERR_ALIGNMENT;
     cudaStream_t s = (cudaStream_t)stream;
+    if (to_sliced)
+        return nq::word64_to_sliced_launch(static_cast<const uint64_t*>(src), bits, rows, cols, static_cast<uint8_t*>(dst), s);
     switch (bits) {
-        case 1: return launch_bits<1>(to_sliced, src, rows, cols, dst, s);
-        case 2: return launch_bits<2>(to_sliced, src, rows, cols, dst, s);
-        case 3: return launch_bits<3>(to_sliced, src, rows, cols, dst, s);
-        case 4: return launch_bits<4>(to_sliced, src, rows, cols, dst, s);
-        case 5: return launch_bits<5>(to_sliced, src, rows, cols, dst, s);
-        case 6: return launch_bits<6>(to_sliced, src, rows, cols, dst, s);
-        case 7: return launch_bits<7>(to_sliced, src, rows, cols, dst, s);
-        default: return launch_bits<8>(to_sliced, src, rows, cols, dst, s);
+        case 1: return launch_from_sliced<1>(src, rows, cols, dst, s);
+        case 2: return launch_from_sliced<2>(src, rows, cols, dst, s);
+        case 3: return launch_from_sliced<3>(src, rows, cols, dst, s);
+        case 4: return launch_from_sliced<4>(src, rows, cols, dst, s);
+        case 5: return launch_from_sliced<5>(src, rows, cols, dst, s);
+        case 6: return launch_from_sliced<6>(src, rows, cols, dst, s);
+        case 7: return launch_from_sliced<7>(src, rows, cols, dst, s);
+        default: return launch_from_sliced<8>(src, rows, cols, dst, s);
     }
 }
 
