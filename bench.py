@@ -606,12 +606,35 @@ def _model_rows(nq, torch, wl, dev, conv_batch):
 
 
 def _run_e2e(nq, torch, sizes, host, state, args, world):
-    """The GEMM sweep fed from pinned host buffers, every GEMM result read back: H2D + kernels + D2H timed."""
+    """The GEMM sweep fed from pinned host buffers, every GEMM result read back: H2D + kernels + D2H timed.  The
+    result copies run on a second stream beside the following kernels; the step ends after the last copy."""
     pinned = {s: {k: torch.from_numpy(host[s][k]).pin_memory() for k in ("W", "X", "mask", "w_scale")} for s in sizes}
-    ybuf = torch.empty((max(sizes), max(sizes)), dtype=torch.bfloat16).pin_memory()
+    ybuf = {s: torch.empty((s, s), dtype=torch.bfloat16).pin_memory() for s in sizes}     # contiguous: plain 1-D copies
     steps = max(1, min(args.steps, args.e2e_steps))
     stream = torch.cuda.current_stream()
     counts = {"h2d": 0, "d2h": 0}
+    # results leave on a copy stream while the next kernels run: two device result buffers per size take turns, a
+    # kernel may only overwrite a buffer once the copy that read it has finished
+    copy_stream = torch.cuda.Stream()
+    ydev = {s: [state[s]["y"], torch.empty_like(state[s]["y"])] for s in sizes}
+    copied = {s: [None, None] for s in sizes}
+    turn = {s: 0 for s in sizes}
+
+    def result_out(s, launch):
+        i = turn[s]
+        turn[s] ^= 1
+        if copied[s][i] is not None:
+            stream.wait_event(copied[s][i])
+        launch(ydev[s][i])
+        done = torch.cuda.Event()
+        done.record(stream)
+        with torch.cuda.stream(copy_stream):
+            copy_stream.wait_event(done)
+            ybuf[s].copy_(ydev[s][i], non_blocking=True)
+            ev = torch.cuda.Event()
+            ev.record(copy_stream)
+        copied[s][i] = ev
+        counts["d2h"] += s * s * 2
 
     def one():
         counts["h2d"] = counts["d2h"] = 0
@@ -624,12 +647,9 @@ def _run_e2e(nq, torch, sizes, host, state, args, world):
                 nq.nq_decompose(d["W"], d["mask"], N_BITS, h, True, out_high=d["hi"][h], out_low=d["lo"][h])
                 nq.nq_drop_low(d["W"], d["lo"][h], N_BITS, h, True, out_high=d["hi"][h])
                 nq.nq_recompose(d["hi"][h], d["lo"][h], s, s, N_BITS, h, True, out=d["w_rec"])
-                nq.nq_gemm_part(d["X"], d["hi"][h], s, N_BITS, h, d["w_scale"], ACT_SCALE, y_out=d["y"])
-                ybuf[:s, :s].copy_(d["y"], non_blocking=True)
-                counts["d2h"] += s * s * 2
-            nq.nq_gemm_full(d["X"], d["w_rec"], d["w_scale"], ACT_SCALE, y_out=d["y"])
-            ybuf[:s, :s].copy_(d["y"], non_blocking=True)
-            counts["d2h"] += s * s * 2
+                result_out(s, lambda y: nq.nq_gemm_part(d["X"], d["hi"][h], s, N_BITS, h, d["w_scale"], ACT_SCALE, y_out=y))
+            result_out(s, lambda y: nq.nq_gemm_full(d["X"], d["w_rec"], d["w_scale"], ACT_SCALE, y_out=y))
+        stream.wait_stream(copy_stream)               # the step ends when its last result is on the host
 
     one()
     torch.cuda.synchronize()
