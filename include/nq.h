@@ -169,8 +169,9 @@ NQ_API int nq_drop_low_batched(const void *table, int count, int64_t work_items,
  *   X (device) int8 [M, K] pitch ldx;  W (device) int8 [N, K] pitch ldw;  both 16-byte aligned with
  *   pitches that are multiples of 16.  w_scale (device) fp32 [N]; bias (device) fp32 [N] or NULL.
  *   acc_out (device, out) int32 [M, N] pitch ld_acc, or NULL.  Y (device, out) [M, N] pitch ldy of
- *   y_dtype, or NULL.  At least one of acc_out, Y must be given.  Y and acc_out 16-byte aligned,
- *   pitches multiples of 4 elements.  K < 2^17 so that the int32 accumulator cannot overflow.
+ *   y_dtype, or NULL.  At least one of acc_out, Y must be given.  Outputs whose base address and row pitch
+ *   (in bytes) are multiples of 16 are written with TMA tile stores; any other element-aligned output takes a
+ *   slower path with ordinary stores (same results).  K < 2^17 so that the int32 accumulator cannot overflow.
  */
 NQ_API int nq_gemm_full(const int8_t *X, int64_t ldx, const int8_t *W, int64_t ldw,
                  const float *w_scale, float act_scale, const float *bias,
