@@ -190,6 +190,24 @@ NQ_API int nq_gemm_part(const int8_t *X, int64_t ldx, const void *packed_high, i
                  int32_t *acc_out, int64_t ld_acc, void *Y, int64_t ldy, int y_dtype, void *stream);
 
 /*
+ * Nested full-bit GEMM -- the full-bit layer computed straight from the two stored parts, with no INT8 copy of
+ * the weights in memory: the kernel rebuilds w_int = w_high * 2^l + w_low (Eq. 5) in shared memory while it
+ * unpacks.  A model then occupies (n + 1) / 8 bytes per weight in full-bit mode and h / 8 in part-bit mode, and
+ * the upgrade is the arrival of w_low alone, the byte model of the paper's switching-overhead analysis.
+ *   acc, Y      exactly those of nq_gemm_full on the tensor nq_recompose would write
+ *   packed_high (device) sliced [N, K] tensor of h_bits fields
+ *   packed_low  (device) sliced [N, K] tensor of (n_bits - h_bits + 1)-bit fields: the COMPENSATED lower-bit
+ *               weights, as nq_decompose writes them with compensate != 0.  For such a pair Eq. 5 is exact and
+ *               stays inside INTn; for other field values the sum wraps modulo 2^n instead of being clipped.
+ *   n_bits 8 with h_bits in [2, 7], or n_bits 6 with h_bits in [2, 5]; anything else NQ_ERR_UNSUPPORTED.
+ *   The other arguments are those of nq_gemm_full.
+ */
+NQ_API int nq_gemm_nested(const int8_t *X, int64_t ldx, const void *packed_high, const void *packed_low,
+                   int n_bits, int h_bits, const float *w_scale, float act_scale, const float *bias,
+                   int64_t M, int64_t N, int64_t K,
+                   int32_t *acc_out, int64_t ld_acc, void *Y, int64_t ldy, int y_dtype, void *stream);
+
+/*
  * Implicit-GEMM convolution on the nested weights, zero padding (the zero-point is 0):
  *   acc[b, p, q, co] = sum_{r, s, ci} x[b, p*stride - pad + r, q*stride - pad + s, ci] * w[co, r, s, ci]
  *   Y = dequantisation as in nq_gemm_full (part_bit == 0) or nq_gemm_part (part_bit != 0).

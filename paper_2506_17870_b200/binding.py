@@ -29,7 +29,7 @@ EXPORTS = (
     "nq_batch_table_bytes", "nq_batch_plan", "nq_recompose_batched", "nq_drop_low_batched",
     "nq_gemm_full", "nq_gemm_part", "nq_conv_workspace_bytes", "nq_conv_implicit_gemm",
     "nq_conv_implicit_gemm_static",
-    "nq_gemm_full_q8", "nq_gemm_part_q8", "nq_conv_implicit_gemm_q8",
+    "nq_gemm_full_q8", "nq_gemm_part_q8", "nq_conv_implicit_gemm_q8", "nq_gemm_nested",
     "nq_device_status",
 )
 
@@ -310,6 +310,25 @@ def nq_gemm_part(X: torch.Tensor, packed_high: torch.Tensor, N: int, n_bits: int
                               ctypes.c_float(act_scale), _ptr(bias), _i64(M), _i64(N), _i64(K), _ptr(acc),
                               _i64(_ld(acc) if acc is not None else 0), _ptr(y), _i64(_ld(y) if y is not None else 0),
                               _y_dtype(y.dtype) if y is not None else NQ_F32, _stream()), "nq_gemm_part")
+    return acc, y
+
+
+def nq_gemm_nested(X: torch.Tensor, packed_high: torch.Tensor, packed_low: torch.Tensor, N: int, n_bits: int,
+                   h_bits: int, w_scale: torch.Tensor, act_scale: float, bias: Optional[torch.Tensor] = None,
+                   want_acc: bool = False, y_dtype=torch.float32, acc_out: Optional[torch.Tensor] = None,
+                   y_out: Optional[torch.Tensor] = None):
+    """Full-bit layer computed from the packed higher-bit and compensated lower-bit tensors (no INT8 copy)."""
+    _need(X, torch.int8, "X", 2)
+    _need(packed_high, torch.uint8, "packed_high")
+    _need(packed_low, torch.uint8, "packed_low")
+    _need(w_scale, torch.float32, "w_scale", 1)
+    M, K = X.shape
+    acc, y = _gemm_outputs(M, N, X.device, want_acc, y_dtype, acc_out, y_out)
+    _check(lib().nq_gemm_nested(_ptr(X), _i64(_ld(X)), _ptr(packed_high), _ptr(packed_low), n_bits, h_bits,
+                                _ptr(w_scale), ctypes.c_float(act_scale), _ptr(bias), _i64(M), _i64(N), _i64(K),
+                                _ptr(acc), _i64(_ld(acc) if acc is not None else 0), _ptr(y),
+                                _i64(_ld(y) if y is not None else 0),
+                                _y_dtype(y.dtype) if y is not None else NQ_F32, _stream()), "nq_gemm_nested")
     return acc, y
 
 

@@ -79,6 +79,9 @@ struct ContractionArgs {
     int packed_stages;   // part-bit: depth of the packed-tile ring (1..kMaxPackedStages)
     const uint8_t* packed_b;   // part-bit: the packed matrix itself and its row pitch in bytes
     long long packed_pitch;
+    const uint8_t* packed_low;   // nested full-bit mode: the packed lower-bit matrix, its row pitch and field width
+    long long low_pitch;
+    int low_bits;
     int32_t* acc_out;
     long long ld_acc;
     void* y;
@@ -179,6 +182,62 @@ __device__ __forceinline__ void expand_packed_unit(const PackedUnit& r, uint32_t
             const uint32_t moved = net >= 0 ? (r.d << net) : (r.d >> (-net));
             T[q] |= moved & (0x80808080u >> used);
         }
+    }
+}
+
+// The same expansion with the field placed SKIP bits below the top of each byte (SKIP + H <= 8).
+template <int H, int SKIP>
+__device__ __forceinline__ void expand_packed_unit_at(const PackedUnit& r, uint32_t (&T)[8]) {
+    static_assert(SKIP >= 0 && SKIP + H <= 8, "field does not fit in a byte");
+#pragma unroll
+    for (int q = 0; q < 8; ++q) T[q] = 0;
+    int used = SKIP;
+    if (H & 4) {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const uint32_t word = (q < 2) ? r.a.x : (q < 4) ? r.a.y : (q < 6) ? r.a.z : r.a.w;
+            const int net = 4 * (q & 1) - used;
+            const uint32_t moved = net >= 0 ? (word << net) : (word >> (-net));
+            T[q] = moved & (0xf0f0f0f0u >> used);
+        }
+        used += 4;
+    }
+    if (H & 2) {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const uint32_t word = (q < 4) ? r.c.x : r.c.y;
+            const int net = 2 * (q & 3) - used;
+            const uint32_t moved = net >= 0 ? (word << net) : (word >> (-net));
+            T[q] |= moved & (0xc0c0c0c0u >> used);
+        }
+        used += 2;
+    }
+    if (H & 1) {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int net = q - used;
+            const uint32_t moved = net >= 0 ? (r.d << net) : (r.d >> (-net));
+            T[q] |= moved & (0x80808080u >> used);
+        }
+    }
+}
+
+// Eq. 5 on 32 fields at once, for INTn weights kept in the top n bits of a byte: T holds w_high * 2^l (the
+// higher-bit field at the top of the byte), L the (l+1)-bit compensated lower-bit field ending at bit 8 - n.
+// The two overlap in one bit, the lower field's sign: w_int = (hi | lo without its sign bit) - sign bit, a
+// per-byte subtraction done on the whole word (bit 7 of every byte is set first so that no borrow crosses a
+// byte, and put right afterwards).  The sum is taken modulo 256: for a compensated decomposition Eq. 5 is exact
+// and stays inside INTn, so the clip of the definition never acts.
+template <int NB, int L1>
+__device__ __forceinline__ void recompose_unit(uint32_t (&T)[8], const uint32_t (&L)[8]) {
+    static_assert(NB - L1 >= 1 && NB - L1 <= 6, "the sign of the lower field must lie below bit 7");
+    constexpr uint32_t SIGN = 0x80808080u >> (NB - L1);
+    constexpr uint32_t TOP = 0x80808080u;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        const uint32_t v = T[q] | (L[q] & ~SIGN);
+        const uint32_t m = L[q] & SIGN;
+        T[q] = ((v | TOP) - m) ^ (~v & TOP);
     }
 }
 
@@ -862,6 +921,6 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
                     const void* Bmat, int64_t ldb, bool part, int n_bits, int h_bits,
                     const float* w_scale, float act_scale, const float* bias, int64_t M, int64_t N, int64_t K,
                     int32_t* acc_out, int64_t ld_acc, void* Y, int64_t ldy, int y_dtype, cudaStream_t stream,
-                    const OutQuant* oq = nullptr);
+                    const OutQuant* oq = nullptr, const void* Blow = nullptr);
 
 }  // namespace nq

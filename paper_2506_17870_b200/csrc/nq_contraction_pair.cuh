@@ -82,9 +82,11 @@ __device__ __forceinline__ void advance_cursor(StageCursor& c, int steps, int k_
 }
 
 // The packed fields of one stage (this CTA's 128 rows of B x one 128-field group) into registers.
-template <int H>
+// L1 > 0 (nested full-bit mode): the L1-bit lower-bit fields of the same weights as well.
+template <int H, int L1>
 __device__ __forceinline__ void fetch_stage(const ContractionArgs& p, const PairUnpackCtx& cx, const StageCursor& c,
-                                            PackedUnit (&raw)[kPairUnitsPerThread]) {
+                                            PackedUnit (&raw)[kPairUnitsPerThread],
+                                            PackedUnit (&raw_low)[L1 > 0 ? kPairUnitsPerThread : 1]) {
     int mt2, nt;
     tile_coords(c.tile, p, mt2, nt);
     const int brow = nt * kPairBN + (int)cx.rank * (kPairBN / 2);
@@ -95,20 +97,32 @@ __device__ __forceinline__ void fetch_stage(const ContractionArgs& p, const Pair
         const int row = brow + (task >> 2);
         fetch_packed_unit<H>(base + (long long)row * p.packed_pitch, task & 3, row < p.N, raw[i]);
     }
+    if (L1 > 0) {
+        const uint8_t* low = p.packed_low + (long long)c.kb * (16 * L1);
+#pragma unroll
+        for (int i = 0; i < kPairUnitsPerThread; ++i) {
+            const int task = i * kUnpackGroupThreads + cx.utid;
+            const int row = brow + (task >> 2);
+            fetch_packed_unit<(L1 > 0 ? L1 : 1)>(low + (long long)row * p.low_pitch, task & 3, row < p.N, raw_low[i]);
+        }
+    }
 }
 
 // One unpack group of the DIRECT variant: for each of its stages wait for the slot, expand the fields fetched a
 // turn earlier into the int8 tile, tell the leader's MMA thread, and only then fetch the fields of its next
 // stage -- they have until the group's next turn to arrive.  (Fetching before the proxy fence was slower.)
-template <int MODE, int H>
+// NB > 0: nested full-bit mode for INT(NB|H) -- the weights are recomposed from both fields (Eq. 5).
+template <int MODE, int H, int NB = 0>
 __device__ __forceinline__ void pair_unpack_direct(const ContractionArgs& p, const PairUnpackCtx& cx) {
     using namespace sm100;
     constexpr int HALF = kPairBN / 2;
     constexpr int B_BYTES = b_stage_bytes(HALF);
+    constexpr int L1 = NB > 0 ? NB - H + 1 : 0;                // compensated lower-bit field: l + 1 bits
     PackedUnit raw[kPairUnitsPerThread];
+    PackedUnit raw_low[L1 > 0 ? kPairUnitsPerThread : 1];
     StageCursor cur{0u, cx.pair, 0};
     advance_cursor(cur, cx.group, p.k_blocks, cx.num_pairs, cx.num_tiles);
-    if (cur.tile < cx.num_tiles) fetch_stage<H>(p, cx, cur, raw);
+    if (cur.tile < cx.num_tiles) fetch_stage<H, L1>(p, cx, cur, raw, raw_low);
     while (cur.tile < cx.num_tiles) {
         const uint32_t s = cur.it % kPairStagesPart, use = cur.it / kPairStagesPart;
         bool ok = mbar_wait_cluster(smem_u32(&cx.empty[s]), (use & 1) ^ 1, cx.abort_flag, p.status, 0x141u);
@@ -120,6 +134,11 @@ __device__ __forceinline__ void pair_unpack_direct(const ContractionArgs& p, con
             const int task = i * kUnpackGroupThreads + cx.utid;
             uint32_t T[8];
             expand_packed_unit<H>(raw[i], T);
+            if (L1 > 0) {
+                uint32_t L[8];
+                expand_packed_unit_at<(L1 > 0 ? L1 : 1), (L1 > 0 ? NB - L1 : 0)>(raw_low[i], L);
+                recompose_unit<(L1 > 0 ? NB : 8), (L1 > 0 ? L1 : 7)>(T, L);
+            }
             store_expanded_unit<HALF, MODE>(dst, task >> 2, task & 3, T);
         }
         fence_proxy_async_smem();
@@ -129,7 +148,7 @@ __device__ __forceinline__ void pair_unpack_direct(const ContractionArgs& p, con
             else signal_remote_tx4(map_to_cta(smem_u32(cx.signal_sink), 0), map_to_cta(smem_u32(&cx.full[s]), 0));
         }
         advance_cursor(cur, kUnpackGroups, p.k_blocks, cx.num_pairs, cx.num_tiles);
-        if (cur.tile < cx.num_tiles) fetch_stage<H>(p, cx, cur, raw);
+        if (cur.tile < cx.num_tiles) fetch_stage<H, L1>(p, cx, cur, raw, raw_low);
     }
 }
 
@@ -139,7 +158,7 @@ __host__ __device__ constexpr int pair_threads(bool part, bool direct) {
     return part ? (direct ? kBaseThreads + kUnpackThreads : kBaseThreads + kUnpackThreads + 32) : kBaseThreads;
 }
 
-template <bool PART, int MODE, bool DIRECT = false>
+template <bool PART, int MODE, bool DIRECT = false, int NEST = 0>
 __global__ void __launch_bounds__(pair_threads(PART, DIRECT), 1)
 contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                         const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmAcc,
@@ -412,11 +431,29 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         cx.group = (warp - kFirstUnpackWarp) / kUnpackGroupWarps;
         cx.utid = (threadIdx.x - kBaseThreads) % kUnpackGroupThreads;
         cx.lane = lane;
-        switch (p.h_bits) {
-            case 1: pair_unpack_direct<MODE, 1>(p, cx); break;
-            case 2: pair_unpack_direct<MODE, 2>(p, cx); break;
-            case 3: pair_unpack_direct<MODE, 3>(p, cx); break;
-            default: pair_unpack_direct<MODE, 4>(p, cx); break;
+        if constexpr (NEST == 8) {
+            switch (p.h_bits) {
+                case 2: pair_unpack_direct<MODE, 2, NEST>(p, cx); break;
+                case 3: pair_unpack_direct<MODE, 3, NEST>(p, cx); break;
+                case 4: pair_unpack_direct<MODE, 4, NEST>(p, cx); break;
+                case 5: pair_unpack_direct<MODE, 5, NEST>(p, cx); break;
+                case 6: pair_unpack_direct<MODE, 6, NEST>(p, cx); break;
+                default: pair_unpack_direct<MODE, 7, NEST>(p, cx); break;
+            }
+        } else if constexpr (NEST == 6) {
+            switch (p.h_bits) {
+                case 2: pair_unpack_direct<MODE, 2, NEST>(p, cx); break;
+                case 3: pair_unpack_direct<MODE, 3, NEST>(p, cx); break;
+                case 4: pair_unpack_direct<MODE, 4, NEST>(p, cx); break;
+                default: pair_unpack_direct<MODE, 5, NEST>(p, cx); break;
+            }
+        } else {
+            switch (p.h_bits) {
+                case 1: pair_unpack_direct<MODE, 1>(p, cx); break;
+                case 2: pair_unpack_direct<MODE, 2>(p, cx); break;
+                case 3: pair_unpack_direct<MODE, 3>(p, cx); break;
+                default: pair_unpack_direct<MODE, 4>(p, cx); break;
+            }
         }
     } else if (PART && warp < kPackedProducerWarp) {
         // ------------------------------------------------------------------ unpackers (both CTAs, own half of B)

@@ -111,7 +111,7 @@ int launch_mode(int mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const 
 }
 
 // CTA-pair kernel: a cluster of two CTAs per 256 x 256 tile
-template <bool PART, int MODE, bool DIRECT = false>
+template <bool PART, int MODE, bool DIRECT = false, int NEST = 0>
 int launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const OutMaps& om, const ContractionArgs& a,
                 cudaStream_t stream) {
     const int smem = pair_smem_bytes(PART, a.h_bits, a.packed_stages);
@@ -119,7 +119,7 @@ int launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const OutMaps& o
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return NQ_ERR_CUDA;
     if (smem > configured[dev]) {
-        if (cudaFuncSetAttribute(contraction_pair_kernel<PART, MODE, DIRECT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(contraction_pair_kernel<PART, MODE, DIRECT, NEST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  smem) != cudaSuccess)
             return NQ_ERR_CUDA;
         configured[dev] = smem;
@@ -139,7 +139,7 @@ int launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const OutMaps& o
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, contraction_pair_kernel<PART, MODE, DIRECT>, tmA, tmB, om.y, om.acc, a) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, contraction_pair_kernel<PART, MODE, DIRECT, NEST>, tmA, tmB, om.y, om.acc, a) != cudaSuccess) {
         (void)cudaGetLastError();
         return NQ_ERR_CUDA;
     }
@@ -205,7 +205,10 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
                     const void* Bmat, int64_t ldb, bool part, int n_bits, int h_bits,
                     const float* w_scale, float act_scale, const float* bias, int64_t M, int64_t N, int64_t K,
                     int32_t* acc_out, int64_t ld_acc, void* Y, int64_t ldy, int y_dtype, cudaStream_t stream,
-                    const OutQuant* oq) {
+                    const OutQuant* oq, const void* Blow) {
+    // Blow given: nested full-bit mode -- Bmat is the packed higher-bit matrix, Blow the packed (l + 1)-bit
+    // lower-bit matrix, and the unpack warps of the pair kernel rebuild w_int from both (GEMM mode only).
+    const bool nest = Blow != nullptr;
     // Tile shape: the widest tile reuses operands best, but a small problem must first of all fill the
     // machine.  Estimate, for each candidate, (waves of tiles over the SMs) x (stages per tile) x (cycles per
     // stage, measured orders of magnitude: narrow tiles are load-bound, the wide single-CTA tile is
@@ -219,9 +222,10 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
         const bool cand_pair[4] = {false, false, false, true};
         const double stage_cycles[4] = {260.0, 330.0, 800.0, 560.0};
         for (int c = 0; c < 4; ++c) {
-            if (cand_pair[c] && (!pairs_enabled() || m_tiles < 2)) continue;
+            if (nest && !cand_pair[c]) continue;
+            if (cand_pair[c] && !nest && (!pairs_enabled() || m_tiles < 2)) continue;
             if (c > 0 && N <= cand_bn[c - 1] && !(c == 3)) continue;          // no wider than the output needs
-            if (c == 3 && N <= 128) continue;
+            if (c == 3 && N <= 128 && !nest) continue;
             const long long nt = (N + cand_bn[c] - 1) / cand_bn[c];
             const long long tiles = (cand_pair[c] ? (m_tiles + 1) / 2 : m_tiles) * nt;
             const long long slots = cand_pair[c] ? sms / 2 : sms;
@@ -254,14 +258,19 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
     bool direct = false;
     if (part) {
         const int l = n_bits - h_bits;
-        a.pow2_l = (float)(1 << l);
-        a.acc_shift = 8 - h_bits;
+        a.pow2_l = nest ? 1.0f : (float)(1 << l);
+        a.acc_shift = nest ? 8 - n_bits : 8 - h_bits;        // nested: w_int sits in the top n bits of the byte
         a.unshift = 1.0f / (float)(1 << a.acc_shift);
         a.h_bits = h_bits;
         // as deep a ring of packed tiles as shared memory allows: it is what hides the load latency of B
         // (pair kernel: a multiple of its unpack group count, see nq_contraction_pair.cuh)
         a.packed_stages = 0;
-        direct = pair && h_bits <= 4 && direct_fetch_enabled();
+        direct = nest || (pair && h_bits <= 4 && direct_fetch_enabled());
+        if (nest) {
+            a.low_bits = l + 1;
+            a.packed_low = static_cast<const uint8_t*>(Blow);
+            a.low_pitch = (long long)((K + 127) / 128) * 16 * a.low_bits;
+        }
         const int step = pair ? kUnpackGroups : 1;
         for (int d = direct ? 0 : kMaxPackedStages; d >= step; d -= step)
             if ((pair ? pair_smem_bytes(true, h_bits, d) : contraction_smem_bytes(bn, true, h_bits, d)) <= kSmemLimit) {
@@ -281,6 +290,11 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
                      : encode_tensor_map_2d(&tmB, Bmat, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, kBK, b_box_rows, 128);
         if (st != NQ_OK) return st;
     }
+    if (nest) {
+        if (mode != kModeGemm || !pair) return NQ_ERR_UNSUPPORTED;
+        return n_bits == 8 ? launch_pair<true, kModeGemm, true, 8>(tmA, tmB, om, a, stream)
+                           : launch_pair<true, kModeGemm, true, 6>(tmA, tmB, om, a, stream);
+    }
     if (pair && direct) return launch_pair_mode<true, true>(mode, tmA, tmB, om, a, stream);
     if (pair) return part ? launch_pair_mode<true>(mode, tmA, tmB, om, a, stream) : launch_pair_mode<false>(mode, tmA, tmB, om, a, stream);
     if (part) {
@@ -298,11 +312,13 @@ namespace {
 int gemm_common(const int8_t* X, int64_t ldx, const void* Bmat, int64_t ldb, bool part, int n_bits, int h_bits,
                 const float* w_scale, float act_scale, const float* bias, int64_t M, int64_t N, int64_t K,
                 int32_t* acc_out, int64_t ld_acc, void* Y, int64_t ldy, int y_dtype, void* stream,
-                const OutQuant* oq = nullptr) {
+                const OutQuant* oq = nullptr, const void* Blow = nullptr) {
     if (M < 0 || N < 0 || K < 0) return NQ_ERR_INVALID_ARG;
     if (y_dtype != NQ_F32 && y_dtype != NQ_BF16 && !(y_dtype == kOutI8 && oq)) return NQ_ERR_INVALID_ARG;
     if (oq && !(oq->out_scale > 0.0f)) return NQ_ERR_INVALID_ARG;
     if (part && (n_bits < 2 || n_bits > 8 || h_bits < 1 || h_bits >= n_bits)) return NQ_ERR_UNSUPPORTED;
+    if (Blow && ((n_bits != 8 && n_bits != 6) || h_bits < 2)) return NQ_ERR_UNSUPPORTED;
+    if (Blow && !aligned16(Blow)) return NQ_ERR_ALIGNMENT;
     if (K >= (1 << 17) || M > (1ll << 30) || N > (1ll << 30)) return NQ_ERR_UNSUPPORTED;
     if (M == 0 || N == 0) return NQ_OK;
     if (!acc_out && !Y) return NQ_ERR_INVALID_ARG;
@@ -318,7 +334,7 @@ int gemm_common(const int8_t* X, int64_t ldx, const void* Bmat, int64_t ldb, boo
     if (st != NQ_OK) return st;
     return run_contraction(tmA, kModeGemm, nullptr, (int)((M + kBM - 1) / kBM), (int)((K + kBK - 1) / kBK), Bmat, ldb,
                            part, n_bits, h_bits, w_scale, act_scale, bias, M, N, K, acc_out, ld_acc, Y, ldy, y_dtype,
-                           (cudaStream_t)stream, oq);
+                           (cudaStream_t)stream, oq, Blow);
 }
 
 }  // namespace
@@ -349,6 +365,14 @@ int nq_gemm_part_q8(const int8_t* X, int64_t ldx, const void* packed_high, int n
     if (!Yq) return NQ_ERR_INVALID_ARG;
     return nq::gemm_common(X, ldx, packed_high, 0, true, n_bits, h_bits, w_scale, act_scale, bias, M, N, K, nullptr, 0, Yq,
                            ldyq, nq::kOutI8, stream, &oq);
+}
+
+int nq_gemm_nested(const int8_t* X, int64_t ldx, const void* packed_high, const void* packed_low, int n_bits, int h_bits,
+                   const float* w_scale, float act_scale, const float* bias, int64_t M, int64_t N, int64_t K,
+                   int32_t* acc_out, int64_t ld_acc, void* Y, int64_t ldy, int y_dtype, void* stream) {
+    if (!packed_low) return (M == 0 || N == 0) && M >= 0 && N >= 0 && K >= 0 ? NQ_OK : NQ_ERR_INVALID_ARG;
+    return nq::gemm_common(X, ldx, packed_high, 0, true, n_bits, h_bits, w_scale, act_scale, bias, M, N, K, acc_out,
+                           ld_acc, Y, ldy, y_dtype, stream, nullptr, packed_low);
 }
 
 int nq_gemm_part(const int8_t* X, int64_t ldx, const void* packed_high, int n_bits, int h_bits, const float* w_scale,
