@@ -349,6 +349,7 @@ def run_ours(args, rank, world, local_rank):
     if model_switch is not None:
         line["rows"]["model_switch"] = model_switch
         line["rows"]["word64_convert_8192"] = _word64_rows(nq, torch, dev)
+        line["rows"]["gemm_nested_8192"] = _nested_rows(nq, torch, dev)
     if model_rows is not None:
         line["rows"].update(model_rows)
     if world == 1 and not args.no_cpu_baseline:
@@ -439,6 +440,41 @@ def _model_switch(nq, torch, wl, dev):
         res["tensors"] = len(shapes)
         res["algorithmic_mb"] = round(nbytes / 1e6, 1)
         out[name] = res
+    return out
+
+
+def _nested_rows(nq, torch, dev):
+    """The full-bit layer computed straight from packed w_high and compensated w_low (no INT8 copy of the weights):
+    8192^3, median of 5 launches per nesting, against the int8 peak; outputs checked equal to the full-bit GEMM's."""
+    peaks = measured_peaks()
+    int8_peak = 2.0 * peaks["bf16_tflops"]
+    S = 8192
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(11)
+    W = torch.randint(-128, 128, (S, S), dtype=torch.int8, device=dev, generator=gen)
+    X = torch.randint(-128, 128, (S, S), dtype=torch.int8, device=dev, generator=gen)
+    mask = torch.randint(0, 2, (S, S), dtype=torch.uint8, device=dev, generator=gen)
+    ws = torch.rand(S, device=dev, generator=gen) * 0.01 + 0.001
+    y = torch.empty((S, S), dtype=torch.float32, device=dev)
+    nq.nq_gemm_full(X, W, ws, ACT_SCALE, y_out=y)
+    ref = y.clone()
+    out = {}
+    for h in HS:
+        hi, lo = nq.nq_decompose(W, mask, N_BITS, h, True)
+        ts = []
+        for rep in range(6):
+            a = torch.cuda.Event(enable_timing=True)
+            b = torch.cuda.Event(enable_timing=True)
+            a.record()
+            nq.nq_gemm_nested(X, hi, lo, S, N_BITS, h, ws, ACT_SCALE, y_out=y)
+            b.record()
+            torch.cuda.synchronize()
+            if rep:
+                ts.append(a.elapsed_time(b))
+        ms = float(np.median(ts))
+        t = 2.0 * S * S * S / (ms * 1e-3) / 1e12
+        out[f"h{h}"] = {"tops": round(t, 1), "frac_int8_peak": round(t / int8_peak, 3), "ms": round(ms, 4),
+                        "weight_bytes_per_element": (N_BITS + 1) / 8, "equals_full_bit": bool(torch.equal(y, ref))}
     return out
 
 

@@ -79,9 +79,9 @@ struct ContractionArgs {
     int packed_stages;   // part-bit: depth of the packed-tile ring (1..kMaxPackedStages)
     const uint8_t* packed_b;   // part-bit: the packed matrix itself and its row pitch in bytes
     long long packed_pitch;
-    const uint8_t* packed_low;   // nested full-bit mode: the packed lower-bit matrix, its row pitch and field width
-    long long low_pitch;
-    int low_bits;
+    int ring_bits;       // pair kernel: field width of the tensor that feeds the packed-tile ring (h_bits in
+                         // part-bit mode; the wider of the two fields in nested full-bit mode, where packed_b
+                         // is the tensor of the narrower one)
     int32_t* acc_out;
     long long ld_acc;
     void* y;

@@ -27,6 +27,11 @@
 // Direct reads lifted h = 4 from 2.40 to 2.93 POP/s at 8192^3; for h >= 5 the narrow slices need two or three
 // small loads per unit and the load/store unit becomes the limit instead (h = 7 fell to 1.7), so those keep the
 // ring.
+// NESTED (full-bit from the two stored parts, Eq. 5): the wider of the two fields (5 to 7 bits) comes through the
+// ring of packed tiles, the narrower one (2 to 4 bits) by direct reads, and the unpack warps add them.  Both
+// through direct reads ran at a third of the tensor rate: 16 small loads and 36 registers of fields in flight
+// per thread spilled, and the reloads sat on the unpack warps' critical path (a block of 18 or 19 warps cannot
+// have more than 96 registers per thread: five warps share each quarter of the register file).
 // Every wait is bounded; every TMA load has a single destination CTA.
 #pragma once
 #include "nq_contraction.cuh"
@@ -82,11 +87,9 @@ __device__ __forceinline__ void advance_cursor(StageCursor& c, int steps, int k_
 }
 
 // The packed fields of one stage (this CTA's 128 rows of B x one 128-field group) into registers.
-// L1 > 0 (nested full-bit mode): the L1-bit lower-bit fields of the same weights as well.
-template <int H, int L1>
+template <int H>
 __device__ __forceinline__ void fetch_stage(const ContractionArgs& p, const PairUnpackCtx& cx, const StageCursor& c,
-                                            PackedUnit (&raw)[kPairUnitsPerThread],
-                                            PackedUnit (&raw_low)[L1 > 0 ? kPairUnitsPerThread : 1]) {
+                                            PackedUnit (&raw)[kPairUnitsPerThread]) {
     int mt2, nt;
     tile_coords(c.tile, p, mt2, nt);
     const int brow = nt * kPairBN + (int)cx.rank * (kPairBN / 2);
@@ -97,32 +100,20 @@ __device__ __forceinline__ void fetch_stage(const ContractionArgs& p, const Pair
         const int row = brow + (task >> 2);
         fetch_packed_unit<H>(base + (long long)row * p.packed_pitch, task & 3, row < p.N, raw[i]);
     }
-    if (L1 > 0) {
-        const uint8_t* low = p.packed_low + (long long)c.kb * (16 * L1);
-#pragma unroll
-        for (int i = 0; i < kPairUnitsPerThread; ++i) {
-            const int task = i * kUnpackGroupThreads + cx.utid;
-            const int row = brow + (task >> 2);
-            fetch_packed_unit<(L1 > 0 ? L1 : 1)>(low + (long long)row * p.low_pitch, task & 3, row < p.N, raw_low[i]);
-        }
-    }
 }
 
 // One unpack group of the DIRECT variant: for each of its stages wait for the slot, expand the fields fetched a
 // turn earlier into the int8 tile, tell the leader's MMA thread, and only then fetch the fields of its next
 // stage -- they have until the group's next turn to arrive.  (Fetching before the proxy fence was slower.)
-// NB > 0: nested full-bit mode for INT(NB|H) -- the weights are recomposed from both fields (Eq. 5).
-template <int MODE, int H, int NB = 0>
+template <int MODE, int H>
 __device__ __forceinline__ void pair_unpack_direct(const ContractionArgs& p, const PairUnpackCtx& cx) {
     using namespace sm100;
     constexpr int HALF = kPairBN / 2;
     constexpr int B_BYTES = b_stage_bytes(HALF);
-    constexpr int L1 = NB > 0 ? NB - H + 1 : 0;                // compensated lower-bit field: l + 1 bits
     PackedUnit raw[kPairUnitsPerThread];
-    PackedUnit raw_low[L1 > 0 ? kPairUnitsPerThread : 1];
     StageCursor cur{0u, cx.pair, 0};
     advance_cursor(cur, cx.group, p.k_blocks, cx.num_pairs, cx.num_tiles);
-    if (cur.tile < cx.num_tiles) fetch_stage<H, L1>(p, cx, cur, raw, raw_low);
+    if (cur.tile < cx.num_tiles) fetch_stage<H>(p, cx, cur, raw);
     while (cur.tile < cx.num_tiles) {
         const uint32_t s = cur.it % kPairStagesPart, use = cur.it / kPairStagesPart;
         bool ok = mbar_wait_cluster(smem_u32(&cx.empty[s]), (use & 1) ^ 1, cx.abort_flag, p.status, 0x141u);
@@ -134,11 +125,6 @@ __device__ __forceinline__ void pair_unpack_direct(const ContractionArgs& p, con
             const int task = i * kUnpackGroupThreads + cx.utid;
             uint32_t T[8];
             expand_packed_unit<H>(raw[i], T);
-            if (L1 > 0) {
-                uint32_t L[8];
-                expand_packed_unit_at<(L1 > 0 ? L1 : 1), (L1 > 0 ? NB - L1 : 0)>(raw_low[i], L);
-                recompose_unit<(L1 > 0 ? NB : 8), (L1 > 0 ? L1 : 7)>(T, L);
-            }
             store_expanded_unit<HALF, MODE>(dst, task >> 2, task & 3, T);
         }
         fence_proxy_async_smem();
@@ -148,7 +134,57 @@ __device__ __forceinline__ void pair_unpack_direct(const ContractionArgs& p, con
             else signal_remote_tx4(map_to_cta(smem_u32(cx.signal_sink), 0), map_to_cta(smem_u32(&cx.full[s]), 0));
         }
         advance_cursor(cur, kUnpackGroups, p.k_blocks, cx.num_pairs, cx.num_tiles);
-        if (cur.tile < cx.num_tiles) fetch_stage<H, L1>(p, cx, cur, raw, raw_low);
+        if (cur.tile < cx.num_tiles) fetch_stage<H>(p, cx, cur, raw);
+    }
+}
+
+// One unpack group of the NESTED variant, INT(NB|H) with the compensated lower field of L1 = NB - H + 1 bits.  The
+// wider field is read from the ring tile in shared memory, the narrower one was fetched from global memory a
+// turn earlier (p.packed_b is that tensor); Eq. 5 joins them and the stage is handed over as in part-bit mode.
+template <int MODE, int H, int NB>
+__device__ __forceinline__ void pair_unpack_nested(const ContractionArgs& p, const PairUnpackCtx& cx, const uint8_t* sP,
+                                                   int packed_bytes, uint64_t* pfull, uint64_t* pempty) {
+    using namespace sm100;
+    constexpr int HALF = kPairBN / 2;
+    constexpr int B_BYTES = b_stage_bytes(HALF);
+    constexpr int L1 = NB - H + 1;
+    constexpr bool HIGH_IN_RING = H > L1;
+    constexpr int RING_BITS = HIGH_IN_RING ? H : L1;
+    constexpr int DIRECT_BITS = HIGH_IN_RING ? L1 : H;
+    static_assert(DIRECT_BITS >= 1 && DIRECT_BITS <= 4 && RING_BITS <= 7, "field widths");
+    PackedUnit raw[kPairUnitsPerThread];
+    StageCursor cur{0u, cx.pair, 0};
+    advance_cursor(cur, cx.group, p.k_blocks, cx.num_pairs, cx.num_tiles);
+    if (cur.tile < cx.num_tiles) fetch_stage<DIRECT_BITS>(p, cx, cur, raw);
+    while (cur.tile < cx.num_tiles) {
+        const uint32_t s = cur.it % kPairStagesPart, use = cur.it / kPairStagesPart;
+        const uint32_t ps = cur.it % p.packed_stages, puse = cur.it / p.packed_stages;
+        bool ok = mbar_wait(smem_u32(&pfull[ps]), puse & 1, cx.abort_flag, p.status, 0x140u) &&
+                  mbar_wait_cluster(smem_u32(&cx.empty[s]), (use & 1) ^ 1, cx.abort_flag, p.status, 0x141u);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        const uint8_t* src = sP + ps * packed_bytes;
+        uint8_t* dst = cx.sB + s * B_BYTES;
+#pragma unroll
+        for (int i = 0; i < kPairUnitsPerThread; ++i) {
+            const int task = i * kUnpackGroupThreads + cx.utid;
+            PackedUnit ring;
+            load_packed_unit<RING_BITS>(src + (task >> 2) * 16 * RING_BITS, task & 3, ring);
+            uint32_t T[8], L[8];
+            expand_packed_unit<H>(HIGH_IN_RING ? ring : raw[i], T);
+            expand_packed_unit_at<L1, NB - L1>(HIGH_IN_RING ? raw[i] : ring, L);
+            recompose_unit<NB, L1>(T, L);
+            store_expanded_unit<HALF, MODE>(dst, task >> 2, task & 3, T);
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (cx.lane == 0) {
+            if (cx.rank == 0) mbar_arrive(smem_u32(&cx.full[s]));
+            else signal_remote_tx4(map_to_cta(smem_u32(cx.signal_sink), 0), map_to_cta(smem_u32(&cx.full[s]), 0));
+            mbar_arrive(smem_u32(&pempty[ps]));
+        }
+        advance_cursor(cur, kUnpackGroups, p.k_blocks, cx.num_pairs, cx.num_tiles);
+        if (cur.tile < cx.num_tiles) fetch_stage<DIRECT_BITS>(p, cx, cur, raw);
     }
 }
 
@@ -176,7 +212,7 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sA = smem;
     uint8_t* sB = sA + STAGES * A_BYTES;
-    const int packed_bytes = PART ? HALF * 16 * p.h_bits : 0;
+    const int packed_bytes = PART ? HALF * 16 * p.ring_bits : 0;
     uint8_t* sP = sB + STAGES * B_BYTES;
     float* sScale = reinterpret_cast<float*>(sP + (PART ? p.packed_stages * packed_bytes : 0));   // [4 warps][BN]
     float* sBias = sScale + 4 * BN;
@@ -290,7 +326,7 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                     if (!(ok = mbar_wait(smem_u32(&pempty[ps]), (puse & 1) ^ 1, abort_flag, p.status, 0x111u))) break;
                     const uint32_t pb = smem_u32(&pfull[ps]);
                     mbar_arrive_expect_tx(pb, packed_bytes);
-                    tma_load_2d(smem_u32(sP + ps * packed_bytes), &tmB, kb * 16 * p.h_bits, brow, pb);
+                    tma_load_2d(smem_u32(sP + ps * packed_bytes), &tmB, kb * 16 * p.ring_bits, brow, pb);
                 }
             }
             if (!ok) {
@@ -431,28 +467,35 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         cx.group = (warp - kFirstUnpackWarp) / kUnpackGroupWarps;
         cx.utid = (threadIdx.x - kBaseThreads) % kUnpackGroupThreads;
         cx.lane = lane;
+        switch (p.h_bits) {
+            case 1: pair_unpack_direct<MODE, 1>(p, cx); break;
+            case 2: pair_unpack_direct<MODE, 2>(p, cx); break;
+            case 3: pair_unpack_direct<MODE, 3>(p, cx); break;
+            default: pair_unpack_direct<MODE, 4>(p, cx); break;
+        }
+    } else if (PART && NEST != 0 && warp < kPackedProducerWarp) {
+        // ------------------------------------------------------------------ unpackers joining both parts (Eq. 5)
+        PairUnpackCtx cx;
+        cx.sB = sB; cx.full = full; cx.empty = empty; cx.signal_sink = signal_sink; cx.abort_flag = abort_flag;
+        cx.rank = rank; cx.pair = pair; cx.num_pairs = num_pairs; cx.num_tiles = num_tiles;
+        cx.group = (warp - kFirstUnpackWarp) / kUnpackGroupWarps;
+        cx.utid = (threadIdx.x - kBaseThreads) % kUnpackGroupThreads;
+        cx.lane = lane;
         if constexpr (NEST == 8) {
             switch (p.h_bits) {
-                case 2: pair_unpack_direct<MODE, 2, NEST>(p, cx); break;
-                case 3: pair_unpack_direct<MODE, 3, NEST>(p, cx); break;
-                case 4: pair_unpack_direct<MODE, 4, NEST>(p, cx); break;
-                case 5: pair_unpack_direct<MODE, 5, NEST>(p, cx); break;
-                case 6: pair_unpack_direct<MODE, 6, NEST>(p, cx); break;
-                default: pair_unpack_direct<MODE, 7, NEST>(p, cx); break;
+                case 2: pair_unpack_nested<MODE, 2, 8>(p, cx, sP, packed_bytes, pfull, pempty); break;
+                case 3: pair_unpack_nested<MODE, 3, 8>(p, cx, sP, packed_bytes, pfull, pempty); break;
+                case 4: pair_unpack_nested<MODE, 4, 8>(p, cx, sP, packed_bytes, pfull, pempty); break;
+                case 5: pair_unpack_nested<MODE, 5, 8>(p, cx, sP, packed_bytes, pfull, pempty); break;
+                case 6: pair_unpack_nested<MODE, 6, 8>(p, cx, sP, packed_bytes, pfull, pempty); break;
+                default: pair_unpack_nested<MODE, 7, 8>(p, cx, sP, packed_bytes, pfull, pempty); break;
             }
         } else if constexpr (NEST == 6) {
             switch (p.h_bits) {
-                case 2: pair_unpack_direct<MODE, 2, NEST>(p, cx); break;
-                case 3: pair_unpack_direct<MODE, 3, NEST>(p, cx); break;
-                case 4: pair_unpack_direct<MODE, 4, NEST>(p, cx); break;
-                default: pair_unpack_direct<MODE, 5, NEST>(p, cx); break;
-            }
-        } else {
-            switch (p.h_bits) {
-                case 1: pair_unpack_direct<MODE, 1>(p, cx); break;
-                case 2: pair_unpack_direct<MODE, 2>(p, cx); break;
-                case 3: pair_unpack_direct<MODE, 3>(p, cx); break;
-                default: pair_unpack_direct<MODE, 4>(p, cx); break;
+                case 2: pair_unpack_nested<MODE, 2, 6>(p, cx, sP, packed_bytes, pfull, pempty); break;
+                case 3: pair_unpack_nested<MODE, 3, 6>(p, cx, sP, packed_bytes, pfull, pempty); break;
+                case 4: pair_unpack_nested<MODE, 4, 6>(p, cx, sP, packed_bytes, pfull, pempty); break;
+                default: pair_unpack_nested<MODE, 5, 6>(p, cx, sP, packed_bytes, pfull, pempty); break;
             }
         }
     } else if (PART && warp < kPackedProducerWarp) {

@@ -114,7 +114,7 @@ int launch_mode(int mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const 
 template <bool PART, int MODE, bool DIRECT = false, int NEST = 0>
 int launch_pair(const CUtensorMap& tmA, const CUtensorMap& tmB, const OutMaps& om, const ContractionArgs& a,
                 cudaStream_t stream) {
-    const int smem = pair_smem_bytes(PART, a.h_bits, a.packed_stages);
+    const int smem = pair_smem_bytes(PART, a.ring_bits, a.packed_stages);
     static int configured[64] = {0};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return NQ_ERR_CUDA;
@@ -207,7 +207,8 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
                     int32_t* acc_out, int64_t ld_acc, void* Y, int64_t ldy, int y_dtype, cudaStream_t stream,
                     const OutQuant* oq, const void* Blow) {
     // Blow given: nested full-bit mode -- Bmat is the packed higher-bit matrix, Blow the packed (l + 1)-bit
-    // lower-bit matrix, and the unpack warps of the pair kernel rebuild w_int from both (GEMM mode only).
+    // lower-bit matrix, and the unpack warps of the pair kernel rebuild w_int from both (GEMM mode only): the
+    // wider field through the ring of packed tiles, the narrower one by direct reads.
     const bool nest = Blow != nullptr;
     // Tile shape: the widest tile reuses operands best, but a small problem must first of all fill the
     // machine.  Estimate, for each candidate, (waves of tiles over the SMs) x (stages per tile) x (cycles per
@@ -265,23 +266,24 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
         // as deep a ring of packed tiles as shared memory allows: it is what hides the load latency of B
         // (pair kernel: a multiple of its unpack group count, see nq_contraction_pair.cuh)
         a.packed_stages = 0;
-        direct = nest || (pair && h_bits <= 4 && direct_fetch_enabled());
-        if (nest) {
-            a.low_bits = l + 1;
-            a.packed_low = static_cast<const uint8_t*>(Blow);
-            a.low_pitch = (long long)((K + 127) / 128) * 16 * a.low_bits;
-        }
+        direct = !nest && pair && h_bits <= 4 && direct_fetch_enabled();
+        const bool high_in_ring = !nest || h_bits > l + 1;
+        const int ring_bits = high_in_ring ? h_bits : l + 1;
+        const int direct_bits = nest ? (high_in_ring ? l + 1 : h_bits) : h_bits;
+        const void* ring_mat = high_in_ring ? Bmat : Blow;
+        const void* direct_mat = nest ? (high_in_ring ? Blow : Bmat) : Bmat;
+        a.ring_bits = ring_bits;
         const int step = pair ? kUnpackGroups : 1;
         for (int d = direct ? 0 : kMaxPackedStages; d >= step; d -= step)
-            if ((pair ? pair_smem_bytes(true, h_bits, d) : contraction_smem_bytes(bn, true, h_bits, d)) <= kSmemLimit) {
+            if ((pair ? pair_smem_bytes(true, ring_bits, d) : contraction_smem_bytes(bn, true, h_bits, d)) <= kSmemLimit) {
                 a.packed_stages = d;
                 break;
             }
         if (a.packed_stages == 0 && !direct) return NQ_ERR_UNSUPPORTED;
-        const uint64_t row_bytes = (uint64_t)((K + 127) / 128) * 16 * h_bits;
-        a.packed_b = static_cast<const uint8_t*>(Bmat);      // read directly by the DIRECT pair kernel
-        a.packed_pitch = (long long)row_bytes;
-        int st = encode_tensor_map_2d(&tmB, Bmat, row_bytes, (uint64_t)N, row_bytes, 16 * h_bits, b_box_rows, 0);
+        const uint64_t row_bytes = (uint64_t)((K + 127) / 128) * 16 * ring_bits;
+        a.packed_b = static_cast<const uint8_t*>(direct_mat);     // read directly by the unpack warps (DIRECT, nested)
+        a.packed_pitch = (long long)((K + 127) / 128) * 16 * direct_bits;
+        int st = encode_tensor_map_2d(&tmB, ring_mat, row_bytes, (uint64_t)N, row_bytes, 16 * ring_bits, b_box_rows, 0);
         if (st != NQ_OK) return st;
     } else {
         a.pow2_l = 1.0f; a.unshift = 1.0f; a.acc_shift = 0; a.h_bits = 0;
@@ -292,8 +294,8 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
     }
     if (nest) {
         if (mode != kModeGemm || !pair) return NQ_ERR_UNSUPPORTED;
-        return n_bits == 8 ? launch_pair<true, kModeGemm, true, 8>(tmA, tmB, om, a, stream)
-                           : launch_pair<true, kModeGemm, true, 6>(tmA, tmB, om, a, stream);
+        return n_bits == 8 ? launch_pair<true, kModeGemm, false, 8>(tmA, tmB, om, a, stream)
+                           : launch_pair<true, kModeGemm, false, 6>(tmA, tmB, om, a, stream);
     }
     if (pair && direct) return launch_pair_mode<true, true>(mode, tmA, tmB, om, a, stream);
     if (pair) return part ? launch_pair_mode<true>(mode, tmA, tmB, om, a, stream) : launch_pair_mode<false>(mode, tmA, tmB, om, a, stream);
