@@ -774,6 +774,8 @@ def main():
     ap.add_argument("--no-model-rows", dest="model_rows", action="store_false",
                     help="skip the ResNet-101-shaped stack and the ViT-B linears (timed after the steps)")
     ap.add_argument("--model-batch", type=int, default=128)
+    ap.add_argument("--nested-only", action="store_true",
+                    help="time only the nested full-bit GEMM rows (8192^3, h in {4..7}) and print them")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -784,6 +786,14 @@ def main():
         line = run_reference(args, rank, world)
         if line is not None:
             print(json.dumps(line), flush=True)
+        return
+
+    if args.nested_only:
+        if rank == 0:
+            import torch
+            import paper_2506_17870_b200 as nq
+            torch.cuda.set_device(local_rank)
+            print(json.dumps({"rows": {"gemm_nested_8192": _nested_rows(nq, torch, torch.device("cuda", local_rank))}}), flush=True)
         return
 
     if world > 1:
