@@ -545,9 +545,9 @@ def _model_rows(nq, torch, wl, dev, conv_batch):
         desc = nq.nq_conv_desc(conv_batch, L.Cin, L.H, L.W, L.Cout, L.R, L.S, L.stride, L.pad, 1)
         w, ws = _device_conv_weights(torch, L, dev, gen)
         m = torch.randint(0, 2, (L.Cout, w.stride(0)), dtype=torch.uint8, device=dev, generator=gen)[:, :L.K]
-        hi, _ = nq.nq_decompose(w, m, N_BITS, CONV_H, True)
+        hi, lo = nq.nq_decompose(w, m, N_BITS, CONV_H, True)
         work_bytes = max(work_bytes, nq.nq_conv_workspace_bytes(desc))
-        prepared.append({"desc": desc, "w": w, "hi": hi, "ws": ws, "x": xs[key], "act": 0.02,
+        prepared.append({"desc": desc, "w": w, "hi": hi, "lo": lo, "ws": ws, "x": xs[key], "act": 0.02,
                          "y": ybuf[:conv_batch * L.Ho * L.Wo * L.Cout].view(conv_batch, L.Ho, L.Wo, L.Cout)})
     work = torch.empty(work_bytes + 2048, dtype=torch.uint8, device=dev)
     for cs in prepared:
@@ -570,6 +570,23 @@ def _model_rows(nq, torch, wl, dev, conv_batch):
                 per_layer.append([a.elapsed_time(b) for a, b in evs])
         ms = float(np.sum(np.median(np.array(per_layer), axis=0)))
         res["part_bit" if part else "full_bit"] = {"ms": round(ms, 3), "tops": round(ops / (ms * 1e-3) / 1e12, 1)}
+    # the full-bit stack again with no INT8 copy of the weights: every layer rebuilds them from the two packed parts
+    per_layer = []
+    for rep in range(4):
+        evs = []
+        for cs in prepared:
+            a = torch.cuda.Event(enable_timing=True)
+            b = torch.cuda.Event(enable_timing=True)
+            a.record()
+            nq.nq_conv_implicit_gemm_nested(cs["x"], cs["hi"], cs["lo"], cs["desc"], cs["ws"], cs["act"], n_bits=N_BITS,
+                                            h_bits=CONV_H, workspace=cs["work"], y_out=cs["y"])
+            b.record()
+            evs.append((a, b))
+        torch.cuda.synchronize()
+        if rep:
+            per_layer.append([a.elapsed_time(b) for a, b in evs])
+    ms = float(np.sum(np.median(np.array(per_layer), axis=0)))
+    res["nested_full_bit"] = {"ms": round(ms, 3), "tops": round(ops / (ms * 1e-3) / 1e12, 1)}
     res.update({"layers": len(layers), "batch": conv_batch, "weights": sum(L.weights for L in layers),
                 "tera_ops_per_pass": round(ops / 1e12, 3)})
     # the same stack in chained form: NHWC int8 activations in, the next layer's INT8 activations out (requantising

@@ -231,6 +231,16 @@ NQ_API int nq_conv_implicit_gemm(const int8_t *X, const void *Wt, int64_t ldw, i
                           void *workspace, int64_t workspace_bytes, void *stream);
 
 /*
+ * The convolution in nested full-bit mode: nq_conv_implicit_gemm's result for part_bit == 0 on the tensor
+ * nq_recompose would write, computed from the two packed parts as in nq_gemm_nested (same operands, same limits
+ * on n_bits / h_bits; both are sliced tensors of the [Cout, K] weight matrix in (r, s, ci) order).
+ */
+NQ_API int nq_conv_implicit_gemm_nested(const int8_t *X, const void *packed_high, const void *packed_low,
+                                 int n_bits, int h_bits, const nq_conv_desc *desc, const float *w_scale,
+                                 float act_scale, const float *bias, int32_t *acc_out, void *Y, int y_dtype,
+                                 void *workspace, int64_t workspace_bytes, void *stream);
+
+/*
  * The same three layers with a requantising epilogue: the output is the next layer's INT8 activations, so layers
  * can be chained on the device and the output traffic is a quarter of fp32.  The paper quantises activations to
  * 8 bits with the uniform quantiser of Eq. 1 (zero-point 0) but does not say how one layer's output becomes the

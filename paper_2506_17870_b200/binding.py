@@ -29,7 +29,7 @@ EXPORTS = (
     "nq_batch_table_bytes", "nq_batch_plan", "nq_recompose_batched", "nq_drop_low_batched",
     "nq_gemm_full", "nq_gemm_part", "nq_conv_workspace_bytes", "nq_conv_implicit_gemm",
     "nq_conv_implicit_gemm_static",
-    "nq_gemm_full_q8", "nq_gemm_part_q8", "nq_conv_implicit_gemm_q8", "nq_gemm_nested",
+    "nq_gemm_full_q8", "nq_gemm_part_q8", "nq_conv_implicit_gemm_q8", "nq_gemm_nested", "nq_conv_implicit_gemm_nested",
     "nq_device_status",
 )
 
@@ -414,6 +414,35 @@ def nq_conv_implicit_gemm(X: torch.Tensor, Wt: torch.Tensor, desc: nq_conv_desc,
                                        ctypes.byref(desc), _ptr(w_scale), ctypes.c_float(act_scale), _ptr(bias),
                                        _ptr(acc), _ptr(y), _y_dtype(y.dtype) if y is not None else NQ_F32,
                                        _ptr(ws), _i64(ws.numel()), _stream()), "nq_conv_implicit_gemm")
+    return acc, y, workspace
+
+
+def nq_conv_implicit_gemm_nested(X: torch.Tensor, packed_high: torch.Tensor, packed_low: torch.Tensor, desc: nq_conv_desc,
+                                 w_scale: torch.Tensor, act_scale: float, n_bits: int = 8, h_bits: int = 6,
+                                 bias: Optional[torch.Tensor] = None, want_acc: bool = False, y_dtype=torch.float32,
+                                 workspace: Optional[torch.Tensor] = None, y_out: Optional[torch.Tensor] = None):
+    """The full-bit convolution computed from the packed higher-bit and compensated lower-bit tensors.
+    -> (acc int32 [B, Ho, Wo, Cout] or None, Y [B, Ho, Wo, Cout] or None, workspace)."""
+    _need(X, torch.int8, "X")
+    _need(packed_high, torch.uint8, "packed_high")
+    _need(packed_low, torch.uint8, "packed_low")
+    _need(w_scale, torch.float32, "w_scale", 1)
+    Ho = (desc.H + 2 * desc.pad - desc.R) // desc.stride + 1
+    Wo = (desc.W + 2 * desc.pad - desc.S) // desc.stride + 1
+    need = nq_conv_workspace_bytes(desc)
+    if need < 0:
+        raise NqError(1, "nq_conv_workspace_bytes")
+    if workspace is None:
+        workspace = torch.empty(max(need, 1024) + 1024, dtype=torch.uint8, device=X.device)
+    off = (-workspace.data_ptr()) % 1024
+    ws = workspace[off:]
+    shape = (desc.B, Ho, Wo, desc.Cout)
+    acc = torch.empty(shape, dtype=torch.int32, device=X.device) if want_acc else None
+    y = y_out if y_out is not None else (torch.empty(shape, dtype=y_dtype, device=X.device) if y_dtype is not None else None)
+    _check(lib().nq_conv_implicit_gemm_nested(_ptr(X), _ptr(packed_high), _ptr(packed_low), n_bits, h_bits,
+                                              ctypes.byref(desc), _ptr(w_scale), ctypes.c_float(act_scale), _ptr(bias),
+                                              _ptr(acc), _ptr(y), _y_dtype(y.dtype) if y is not None else NQ_F32,
+                                              _ptr(ws), _i64(ws.numel()), _stream()), "nq_conv_implicit_gemm_nested")
     return acc, y, workspace
 
 

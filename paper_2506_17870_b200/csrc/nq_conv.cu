@@ -220,8 +220,11 @@ int64_t nq_conv_workspace_bytes(const nq_conv_desc* d) {
 static int conv_common(const int8_t* X, const void* Wt, int64_t ldw, int part_bit, int n_bits, int h_bits,
                        const nq_conv_desc* d, const float* w_scale, float act_scale, const float* bias,
                        int32_t* acc_out, void* Y, int y_dtype, void* workspace, int64_t workspace_bytes, void* stream_,
-                       const nq::OutQuant* oq) {
+                       const nq::OutQuant* oq, const void* Wlow = nullptr) {
     using namespace nq;
+    // Wlow given: nested full-bit mode -- Wt is the packed higher-bit tensor, Wlow the packed compensated lower-bit one
+    if (Wlow && ((n_bits != 8 && n_bits != 6) || h_bits < 2 || h_bits >= n_bits)) return NQ_ERR_UNSUPPORTED;
+    if (Wlow && !aligned16(Wlow)) return NQ_ERR_ALIGNMENT;
     if (!desc_ok(d)) return NQ_ERR_INVALID_ARG;
     if (y_dtype != NQ_F32 && y_dtype != NQ_BF16 && !(y_dtype == kOutI8 && oq)) return NQ_ERR_INVALID_ARG;
     if (oq && !(oq->out_scale > 0.0f)) return NQ_ERR_INVALID_ARG;
@@ -255,7 +258,7 @@ static int conv_common(const int8_t* X, const void* Wt, int64_t ldw, int part_bi
         if (st != NQ_OK) return st;
         return run_contraction(tmA, kModeGemm, nullptr, (int)((M + kBM - 1) / kBM), (int)((K + kBK - 1) / kBK), Wt, ldw,
                                part_bit != 0, n_bits, h_bits, w_scale, act_scale, bias, M, N, K, acc_out, N, Y, N, y_dtype,
-                               stream, oq);
+                               stream, oq, Wlow);
     }
 
     const int8_t* x_nhwc = X;
@@ -288,7 +291,7 @@ static int conv_common(const int8_t* X, const void* Wt, int64_t ldw, int part_bi
     }
     if (st != NQ_OK) return st;
     return run_contraction(tmA, mode, &g, m_tiles, k_blocks, Wt, ldw, part_bit != 0, n_bits, h_bits, w_scale, act_scale,
-                           bias, M, N, K, acc_out, N, Y, N, y_dtype, stream, oq);
+                           bias, M, N, K, acc_out, N, Y, N, y_dtype, stream, oq, Wlow);
 }
 
 int nq_conv_implicit_gemm(const int8_t* X, const void* Wt, int64_t ldw, int part_bit, int n_bits, int h_bits,
@@ -297,6 +300,16 @@ int nq_conv_implicit_gemm(const int8_t* X, const void* Wt, int64_t ldw, int part
     if (y_dtype != NQ_F32 && y_dtype != NQ_BF16) return NQ_ERR_INVALID_ARG;
     return conv_common(X, Wt, ldw, part_bit, n_bits, h_bits, d, w_scale, act_scale, bias, acc_out, Y, y_dtype, workspace,
                        workspace_bytes, stream, nullptr);
+}
+
+int nq_conv_implicit_gemm_nested(const int8_t* X, const void* packed_high, const void* packed_low, int n_bits, int h_bits,
+                                 const nq_conv_desc* d, const float* w_scale, float act_scale, const float* bias,
+                                 int32_t* acc_out, void* Y, int y_dtype, void* workspace, int64_t workspace_bytes,
+                                 void* stream) {
+    if (y_dtype != NQ_F32 && y_dtype != NQ_BF16) return NQ_ERR_INVALID_ARG;
+    if (!packed_low) return NQ_ERR_INVALID_ARG;
+    return conv_common(X, packed_high, 0, 1, n_bits, h_bits, d, w_scale, act_scale, bias, acc_out, Y, y_dtype, workspace,
+                       workspace_bytes, stream, nullptr, packed_low);
 }
 
 int nq_conv_implicit_gemm_q8(const int8_t* X, const void* Wt, int64_t ldw, int part_bit, int n_bits, int h_bits,

@@ -207,7 +207,7 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
                     int32_t* acc_out, int64_t ld_acc, void* Y, int64_t ldy, int y_dtype, cudaStream_t stream,
                     const OutQuant* oq, const void* Blow) {
     // Blow given: nested full-bit mode -- Bmat is the packed higher-bit matrix, Blow the packed (l + 1)-bit
-    // lower-bit matrix, and the unpack warps of the pair kernel rebuild w_int from both (GEMM mode only): the
+    // lower-bit matrix, and the unpack warps of the pair kernel rebuild w_int from both: the
     // wider field through the ring of packed tiles, the narrower one by direct reads.
     const bool nest = Blow != nullptr;
     // Tile shape: the widest tile reuses operands best, but a small problem must first of all fill the
@@ -293,7 +293,13 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
         if (st != NQ_OK) return st;
     }
     if (nest) {
-        if (mode != kModeGemm || !pair) return NQ_ERR_UNSUPPORTED;
+        if (!pair) return NQ_ERR_UNSUPPORTED;
+        if (mode == kModeConv128)
+            return n_bits == 8 ? launch_pair<true, kModeConv128, false, 8>(tmA, tmB, om, a, stream)
+                               : launch_pair<true, kModeConv128, false, 6>(tmA, tmB, om, a, stream);
+        if (mode == kModeConv64)
+            return n_bits == 8 ? launch_pair<true, kModeConv64, false, 8>(tmA, tmB, om, a, stream)
+                               : launch_pair<true, kModeConv64, false, 6>(tmA, tmB, om, a, stream);
         return n_bits == 8 ? launch_pair<true, kModeGemm, false, 8>(tmA, tmB, om, a, stream)
                            : launch_pair<true, kModeGemm, false, 6>(tmA, tmB, om, a, stream);
     }

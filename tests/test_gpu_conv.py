@@ -52,6 +52,14 @@ def run_layer(L, batch, seed, n=8, h=6, nchw=True, check_y=True):
         assert np.array_equal(got, ref), (L, part, int(np.count_nonzero(got != ref)))
         if check_y:
             assert np.array_equal(host(y), oracle.dequant(ref, ws, sa, (n - h) if part else 0))
+    if n in (6, 8) and h >= 2:
+        # nested full-bit mode: the same full-bit result straight from the two packed parts
+        ref = oracle.conv_acc(X, oracle.recompose(wh, wlo, n, h), L.stride, L.pad).transpose(0, 2, 3, 1)
+        acc, y, _ = nq.nq_conv_implicit_gemm_nested(x_dev, hi, lo, desc, wsd, sa, n_bits=n, h_bits=h, want_acc=True)
+        nq.nq_device_status()
+        assert np.array_equal(host(acc), ref), (L, "nested")
+        if check_y:
+            assert np.array_equal(host(y), oracle.dequant(ref, ws, sa, 0))
 
 
 C = wl.ConvLayer
