@@ -49,8 +49,8 @@ CONV_H = 6
 # a gigabyte per launch): it is taken as four times 8192, every operand and the output growing fourfold.  Must be set
 # to None again when the contraction kernels change.
 NCU_GEMM_DRAM_MB = {
-    4096: {4: 26.2, 5: 27.7, 6: 29.9, 7: 32.3, 0: 34.4},
-    8192: {4: 281.0, 5: 287.0, 6: 310.0, 7: 342.0, 0: 358.0},
+    4096: {4: 25.7, 5: 27.7, 6: 29.9, 7: 32.2, 0: 34.3},
+    8192: {4: 302.0, 5: 285.0, 6: 308.0, 7: 339.0, 0: 349.0},
 }
 
 
