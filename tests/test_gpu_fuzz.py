@@ -48,7 +48,31 @@ def test_random_shapes_both_modes(seed):
                 assert np.array_equal(y.view(torch.int16).cpu().numpy().view(np.uint16), oracle.f32_to_bf16_bits(yref))
             else:
                 assert np.array_equal(y.cpu().numpy(), yref), (M, N, K, h, part)
+        if h >= 2:
+            # nested full-bit mode: the full-bit result again, rebuilt from the two packed parts
+            acc, y = nq.nq_gemm_nested(Xd, hi, lo, N, 8, h, wsd, d["act_scale"], want_acc=True, y_dtype=ydt)
+            ref = oracle.gemm_acc(d["X"], oracle.recompose(wh, wlo, 8, h))
+            assert np.array_equal(acc.cpu().numpy(), ref), (M, N, K, h, "nested")
+            if not bf16:
+                assert np.array_equal(y.cpu().numpy(), oracle.dequant(ref, d["w_scale"], d["act_scale"], 0)), (M, N, K, h)
         nq.nq_device_status()
+
+
+@pytest.mark.parametrize("h", [3, 5, 6])
+def test_repeated_nested_launches_give_identical_bytes(h):
+    M, N, K = 2304, 2048, 3072
+    g = torch.Generator(device="cuda")
+    g.manual_seed(40 + h)
+    X = torch.randint(-128, 128, (M, K), dtype=torch.int8, device="cuda", generator=g)
+    W = torch.randint(-128, 128, (N, K), dtype=torch.int8, device="cuda", generator=g)
+    mask = torch.randint(0, 2, (N, K), dtype=torch.uint8, device="cuda", generator=g)
+    hi, lo = nq.nq_decompose(W, mask, 8, h, True)
+    ws = torch.rand(N, device="cuda", generator=g) * 1e-2 + 1e-3
+    first_f, _ = nq.nq_gemm_full(X, W, ws, 0.05, want_acc=True, y_dtype=None)
+    for _ in range(15):
+        again, _ = nq.nq_gemm_nested(X, hi, lo, N, 8, h, ws, 0.05, want_acc=True, y_dtype=None)
+        assert torch.equal(again, first_f)
+    nq.nq_device_status()
 
 
 @pytest.mark.parametrize("h", [4, 6, 7])
