@@ -19,14 +19,16 @@
 //   tfull[b]   likewise (accumulator b complete)
 //   tempty[b]  lives in the leader: its own epilogue warps arrive, the partner's send 4 announced bytes each
 //   pfull / pempty  packed-tile ring, private to each CTA
-// DIRECT (part-bit, h <= 4): the packed fields never pass through shared memory; each unpack thread reads its
+// DIRECT (part-bit, h = 1, 2, 4): the packed fields never pass through shared memory; each unpack thread reads its
 // fields straight from the packed matrix into registers, one turn ahead of their use.  Reason, measured: the
 // shared-memory port carries per stage and SM 32 KB of operand reads, 16 KB of A, 16 KB of expanded B and the
 // packed tile twice (in by TMA, out to the unpack warps), 64 + 4h KB against 64 KB in the stage's 512 tensor
 // cycles, and the part-bit rate followed that sum (0.80 / 0.76 / 0.73 / 0.70 of the full-bit rate for h = 4 .. 7).
 // Direct reads lifted h = 4 from 2.40 to 2.93 POP/s at 8192^3; for h >= 5 the narrow slices need two or three
 // small loads per unit and the load/store unit becomes the limit instead (h = 7 fell to 1.7), so those keep the
-// ring.
+// ring, and so does h = 3 (two loads: 2.71 against 3.14 POP/s).  Tried for h >= 5 and dropped: the 4-bit slice by
+// direct reads and only the narrow slices through the ring (2.52 / 2.41 / 1.93 against 2.76 / 2.72 / 2.34, same
+// box) -- a direct read exposes the latency of global memory to the unpack warps, the ring's TMA loads run ahead.
 // NESTED (full-bit from the two stored parts, Eq. 5): the wider of the two fields (5 to 7 bits) comes through the
 // ring of packed tiles, the narrower one (2 to 4 bits) by direct reads, and the unpack warps add them.  Both
 // through direct reads ran at a third of the tensor rate: 16 small loads and 36 registers of fields in flight

@@ -129,11 +129,11 @@ def test_full_equals_shifted_part_plus_low_contribution():
     assert torch.equal(full.long(), (part.long() << 3) + low.long())
 
 
-@pytest.mark.parametrize("h", [1, 2, 3, 4])
+@pytest.mark.parametrize("h", [1, 2, 3, 4, 5, 6, 7])
 def test_wide_ragged_gemm_narrow_fields(h, monkeypatch):
-    """Large enough for the CTA-pair kernel, whose unpack warps read fields of at most 4 bits straight from the
-    packed matrix: ragged in M, N and K, checked against the oracle, and bit for bit against the same launch
-    fed through the shared-memory ring of packed tiles."""
+    """Large enough for the CTA-pair kernel, whose unpack warps read fields of 1, 2 and 4 bits straight from the
+    packed matrix: ragged in M, N and K, every width checked against the oracle, and bit for bit against the same
+    launch with every width fed through the shared-memory ring of packed tiles."""
     M, N, K = 3500, 1100, 1100
     d = wl.gemm_inputs(89, h, M, N, K)
     wh, _ = oracle.decompose(d["W"], d["mask"], 8, h, True)
