@@ -126,3 +126,10 @@ def test_unsupported_nestings_and_empty_problems():
             nq.nq_gemm_nested(X, p, p, 16, n, h, ws, 1.0)
     acc, y = nq.nq_gemm_nested(X[:0], p, p, 16, 8, 4, ws, 1.0, want_acc=True)
     assert acc.shape == (0, 16) and y.shape == (0, 16)
+    # a packed operand that is not 16-byte aligned is refused before anything is launched
+    big = torch.zeros(16 * 16 * 9 + 16, dtype=torch.uint8, device="cuda")
+    off = (-big.data_ptr()) % 16 + 4
+    skew = big[off:off + 16 * 16 * 5].view(16, 80)
+    with pytest.raises(nq.NqError):
+        nq.nq_gemm_nested(X, p[:, :64].contiguous(), skew, 16, 8, 4, ws, 1.0)
+    nq.nq_device_status()
