@@ -79,9 +79,12 @@ struct ContractionArgs {
     int packed_stages;   // part-bit: depth of the packed-tile ring (1..kMaxPackedStages)
     const uint8_t* packed_b;   // part-bit: the packed matrix itself and its row pitch in bytes
     long long packed_pitch;
-    int ring_bits;       // pair kernel: field width of the tensor that feeds the packed-tile ring (h_bits in
-                         // part-bit mode; the wider of the two fields in nested full-bit mode, where packed_b
-                         // is the tensor of the narrower one)
+    int ring_bits;       // pair kernel: bits per field in a packed-ring tile (h_bits in part-bit mode; in nested
+                         // full-bit mode the wider of the two fields, plus one when ring2 is set; packed_b is then
+                         // the tensor of the narrower field)
+    int ring_x_bytes;    // ... bytes per 128-field group of the tensor behind tmB
+    int ring2;           // nested mode, 3-bit narrow field: its 1-bit slice is loaded into the ring tile as well,
+                         // through the map passed in the tmAcc slot (accumulators then take ordinary stores)
     int32_t* acc_out;
     long long ld_acc;
     void* y;

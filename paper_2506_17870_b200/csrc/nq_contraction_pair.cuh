@@ -89,13 +89,14 @@ __device__ __forceinline__ void advance_cursor(StageCursor& c, int steps, int k_
 }
 
 // The packed fields of one stage (this CTA's 128 rows of B x one 128-field group) into registers.
-template <int H>
+// GROUP_BITS > H: only the leading H bits' worth of slices of a tensor of GROUP_BITS-bit fields (they start the group).
+template <int H, int GROUP_BITS = H>
 __device__ __forceinline__ void fetch_stage(const ContractionArgs& p, const PairUnpackCtx& cx, const StageCursor& c,
                                             PackedUnit (&raw)[kPairUnitsPerThread]) {
     int mt2, nt;
     tile_coords(c.tile, p, mt2, nt);
     const int brow = nt * kPairBN + (int)cx.rank * (kPairBN / 2);
-    const uint8_t* base = p.packed_b + (long long)c.kb * (16 * H);
+    const uint8_t* base = p.packed_b + (long long)c.kb * (16 * GROUP_BITS);
 #pragma unroll
     for (int i = 0; i < kPairUnitsPerThread; ++i) {
         const int task = i * kUnpackGroupThreads + cx.utid;
@@ -154,10 +155,15 @@ __device__ __forceinline__ void pair_unpack_nested(const ContractionArgs& p, con
     constexpr int RING_BITS = HIGH_IN_RING ? H : L1;
     constexpr int DIRECT_BITS = HIGH_IN_RING ? L1 : H;
     static_assert(DIRECT_BITS >= 1 && DIRECT_BITS <= 4 && RING_BITS <= 7, "field widths");
+    // A 3-bit narrow field would take two small loads per unit (measured a third slower than one): its 1-bit slice
+    // rides in the ring tile instead, behind the wide field's rows (a second tile load, 16 bytes a row), and only
+    // its 2-bit slice is fetched directly.
+    constexpr bool BIT_IN_RING = DIRECT_BITS == 3;
+    constexpr int FETCH_BITS = BIT_IN_RING ? 2 : DIRECT_BITS;
     PackedUnit raw[kPairUnitsPerThread];
     StageCursor cur{0u, cx.pair, 0};
     advance_cursor(cur, cx.group, p.k_blocks, cx.num_pairs, cx.num_tiles);
-    if (cur.tile < cx.num_tiles) fetch_stage<DIRECT_BITS>(p, cx, cur, raw);
+    if (cur.tile < cx.num_tiles) fetch_stage<FETCH_BITS, DIRECT_BITS>(p, cx, cur, raw);
     while (cur.tile < cx.num_tiles) {
         const uint32_t s = cur.it % kPairStagesPart, use = cur.it / kPairStagesPart;
         const uint32_t ps = cur.it % p.packed_stages, puse = cur.it / p.packed_stages;
@@ -172,9 +178,12 @@ __device__ __forceinline__ void pair_unpack_nested(const ContractionArgs& p, con
             const int task = i * kUnpackGroupThreads + cx.utid;
             PackedUnit ring;
             load_packed_unit<RING_BITS>(src + (task >> 2) * 16 * RING_BITS, task & 3, ring);
+            PackedUnit narrow = raw[i];
+            if (BIT_IN_RING)
+                narrow.d = *reinterpret_cast<const uint32_t*>(src + HALF * 16 * RING_BITS + (task >> 2) * 16 + (task & 3) * 4);
             uint32_t T[8], L[8];
-            expand_packed_unit<H>(HIGH_IN_RING ? ring : raw[i], T);
-            expand_packed_unit_at<L1, NB - L1>(HIGH_IN_RING ? raw[i] : ring, L);
+            expand_packed_unit<H>(HIGH_IN_RING ? ring : narrow, T);
+            expand_packed_unit_at<L1, NB - L1>(HIGH_IN_RING ? narrow : ring, L);
             recompose_unit<NB, L1>(T, L);
             store_expanded_unit<HALF, MODE>(dst, task >> 2, task & 3, T);
         }
@@ -186,7 +195,7 @@ __device__ __forceinline__ void pair_unpack_nested(const ContractionArgs& p, con
             mbar_arrive(smem_u32(&pempty[ps]));
         }
         advance_cursor(cur, kUnpackGroups, p.k_blocks, cx.num_pairs, cx.num_tiles);
-        if (cur.tile < cx.num_tiles) fetch_stage<DIRECT_BITS>(p, cx, cur, raw);
+        if (cur.tile < cx.num_tiles) fetch_stage<FETCH_BITS, DIRECT_BITS>(p, cx, cur, raw);
     }
 }
 
@@ -254,7 +263,7 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         prefetch_tensormap(&tmA);
         prefetch_tensormap(&tmB);
         if (p.y_tma) prefetch_tensormap(&tmY);
-        if (p.acc_tma) prefetch_tensormap(&tmAcc);
+        if (p.acc_tma || (NEST != 0 && p.ring2)) prefetch_tensormap(&tmAcc);
     }
     if (warp == 1) {
         tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS);
@@ -328,7 +337,9 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                     if (!(ok = mbar_wait(smem_u32(&pempty[ps]), (puse & 1) ^ 1, abort_flag, p.status, 0x111u))) break;
                     const uint32_t pb = smem_u32(&pfull[ps]);
                     mbar_arrive_expect_tx(pb, packed_bytes);
-                    tma_load_2d(smem_u32(sP + ps * packed_bytes), &tmB, kb * 16 * p.ring_bits, brow, pb);
+                    tma_load_2d(smem_u32(sP + ps * packed_bytes), &tmB, kb * p.ring_x_bytes, brow, pb);
+                    if (NEST != 0 && p.ring2)     // the 1-bit slice of a 3-bit narrow field (tmAcc is its map here)
+                        tma_load_2d(smem_u32(sP + ps * packed_bytes + HALF * p.ring_x_bytes), &tmAcc, kb * 48 + 32, brow, pb);
                 }
             }
             if (!ok) {

@@ -274,10 +274,20 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
         const int direct_bits = nest ? (high_in_ring ? l + 1 : h_bits) : h_bits;
         const void* ring_mat = high_in_ring ? Bmat : Blow;
         const void* direct_mat = nest ? (high_in_ring ? Blow : Bmat) : Bmat;
-        a.ring_bits = ring_bits;
+        const bool ring2 = nest && direct_bits == 3;
+        a.ring2 = ring2 ? 1 : 0;
+        a.ring_bits = ring_bits + (ring2 ? 1 : 0);
+        a.ring_x_bytes = 16 * ring_bits;
+        if (ring2) {
+            // the narrow tensor's 1-bit slice: 16 bytes per row and group, at byte 32 of every 48-byte group
+            const uint64_t nrow = (uint64_t)((K + 127) / 128) * 48;
+            int st2 = encode_tensor_map_2d(&om.acc, direct_mat, nrow, (uint64_t)N, nrow, 16, b_box_rows, 0);
+            if (st2 != NQ_OK) return st2;
+            a.acc_tma = 0;
+        }
         const int step = pair ? kUnpackGroups : 1;
         for (int d = direct ? 0 : kMaxPackedStages; d >= step; d -= step)
-            if ((pair ? pair_smem_bytes(true, ring_bits, d) : contraction_smem_bytes(bn, true, h_bits, d)) <= kSmemLimit) {
+            if ((pair ? pair_smem_bytes(true, a.ring_bits, d) : contraction_smem_bytes(bn, true, h_bits, d)) <= kSmemLimit) {
                 a.packed_stages = d;
                 break;
             }
