@@ -30,7 +30,9 @@
 // direct reads and only the narrow slices through the ring (2.52 / 2.41 / 1.93 against 2.76 / 2.72 / 2.34, same
 // box) -- a direct read exposes the latency of global memory to the unpack warps, the ring's TMA loads run ahead.
 // NESTED (full-bit from the two stored parts, Eq. 5): the wider of the two fields (5 to 7 bits) comes through the
-// ring of packed tiles, the narrower one (2 to 4 bits) by direct reads, and the unpack warps add them.  Both
+// ring of packed tiles, the narrower one (2 to 4 bits) by direct reads -- except the 1-bit slice of a 3-bit narrow
+// field, which is loaded into the ring tile behind the wide field's rows, so that every unit needs one direct
+// load -- and the unpack warps add them.  Both
 // through direct reads ran at a third of the tensor rate: 16 small loads and 36 registers of fields in flight
 // per thread spilled, and the reloads sat on the unpack warps' critical path (a block of 18 or 19 warps cannot
 // have more than 96 registers per thread: five warps share each quarter of the register file).
