@@ -262,6 +262,17 @@ NQ_API int nq_conv_implicit_gemm_q8(const int8_t *X, const void *Wt, int64_t ldw
                              float out_scale, int relu, int8_t *Yq,
                              void *workspace, int64_t workspace_bytes, void *stream);
 
+/* The nested full-bit layers (nq_gemm_nested, nq_conv_implicit_gemm_nested) with the same requantising epilogue. */
+NQ_API int nq_gemm_nested_q8(const int8_t *X, int64_t ldx, const void *packed_high, const void *packed_low,
+                      int n_bits, int h_bits, const float *w_scale, float act_scale, const float *bias,
+                      float out_scale, int relu, int64_t M, int64_t N, int64_t K,
+                      int8_t *Yq, int64_t ldyq, void *stream);
+NQ_API int nq_conv_implicit_gemm_nested_q8(const int8_t *X, const void *packed_high, const void *packed_low,
+                                    int n_bits, int h_bits, const nq_conv_desc *desc, const float *w_scale,
+                                    float act_scale, const float *bias, float out_scale, int relu, int8_t *Yq,
+                                    void *workspace, int64_t workspace_bytes, void *stream);
+
+
 /*
  * The convolution again, for callers that must not allocate.  (The paper has no counterpart; this is a
  * convenience of the library.)  nq_conv_implicit_gemm needs a workspace whenever it re-lays the input

@@ -10,6 +10,7 @@ from .binding import (  # noqa: F401
     nq_drop_low_batched, nq_gemm_full, nq_gemm_part, nq_low_bits, nq_pack, nq_packed_bytes,
     nq_packed_row_bytes, nq_recompose, nq_recompose_batched, nq_tensor_desc, nq_unpack, status_str,
     nq_word64_row_words, nq_word64_to_sliced, nq_sliced_to_word64,
-    nq_gemm_full_q8, nq_gemm_part_q8, nq_conv_implicit_gemm_q8, nq_gemm_nested, nq_conv_implicit_gemm_nested,
+    nq_gemm_full_q8, nq_gemm_part_q8, nq_conv_implicit_gemm_q8, nq_gemm_nested, nq_conv_implicit_gemm_nested, nq_gemm_nested_q8,
+    nq_conv_implicit_gemm_nested_q8,
     nq_rounding_mask, NQ_ROUND_DOWN, NQ_ROUND_UP, NQ_ROUND_NEAREST,
 )

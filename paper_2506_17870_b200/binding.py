@@ -29,7 +29,8 @@ EXPORTS = (
     "nq_batch_table_bytes", "nq_batch_plan", "nq_recompose_batched", "nq_drop_low_batched",
     "nq_gemm_full", "nq_gemm_part", "nq_conv_workspace_bytes", "nq_conv_implicit_gemm",
     "nq_conv_implicit_gemm_static",
-    "nq_gemm_full_q8", "nq_gemm_part_q8", "nq_conv_implicit_gemm_q8", "nq_gemm_nested", "nq_conv_implicit_gemm_nested",
+    "nq_gemm_full_q8", "nq_gemm_part_q8", "nq_conv_implicit_gemm_q8", "nq_gemm_nested", "nq_conv_implicit_gemm_nested", "nq_gemm_nested_q8",
+    "nq_conv_implicit_gemm_nested_q8",
     "nq_device_status",
 )
 
@@ -376,6 +377,42 @@ def nq_conv_implicit_gemm_q8(X: torch.Tensor, Wt: torch.Tensor, desc: nq_conv_de
                                           ctypes.c_float(out_scale), int(bool(relu)), _ptr(y),
                                           ctypes.c_void_p(workspace.data_ptr() + off), _i64(workspace.numel() - off),
                                           _stream()), "nq_conv_implicit_gemm_q8")
+    return y
+
+
+def nq_gemm_nested_q8(X: torch.Tensor, packed_high: torch.Tensor, packed_low: torch.Tensor, N: int, n_bits: int,
+                      h_bits: int, w_scale: torch.Tensor, act_scale: float, out_scale: float, relu: bool = True,
+                      bias: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Nested full-bit layer whose output is the next layer's INT8 activations."""
+    _need(X, torch.int8, "X", 2); _need(packed_high, torch.uint8, "packed_high"); _need(packed_low, torch.uint8, "packed_low")
+    _need(w_scale, torch.float32, "w_scale", 1)
+    M, K = X.shape
+    y = torch.empty((M, N), dtype=torch.int8, device=X.device)
+    _check(lib().nq_gemm_nested_q8(_ptr(X), _i64(_ld(X)), _ptr(packed_high), _ptr(packed_low), n_bits, h_bits,
+                                   _ptr(w_scale), ctypes.c_float(act_scale), _ptr(bias), ctypes.c_float(out_scale),
+                                   int(bool(relu)), _i64(M), _i64(N), _i64(K), _ptr(y), _i64(N), _stream()),
+           "nq_gemm_nested_q8")
+    return y
+
+
+def nq_conv_implicit_gemm_nested_q8(X: torch.Tensor, packed_high: torch.Tensor, packed_low: torch.Tensor,
+                                    desc: nq_conv_desc, w_scale: torch.Tensor, act_scale: float, out_scale: float,
+                                    relu: bool = True, n_bits: int = 8, h_bits: int = 6,
+                                    bias: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                                    y_out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Nested full-bit convolution whose NHWC output is the next layer's INT8 activations."""
+    Ho = (desc.H + 2 * desc.pad - desc.R) // desc.stride + 1
+    Wo = (desc.W + 2 * desc.pad - desc.S) // desc.stride + 1
+    need = nq_conv_workspace_bytes(desc)
+    if workspace is None:
+        workspace = torch.empty(max(need, 0) + 2048, dtype=torch.uint8, device=X.device)
+    off = (-workspace.data_ptr()) % 1024
+    y = y_out if y_out is not None else torch.empty((desc.B, Ho, Wo, desc.Cout), dtype=torch.int8, device=X.device)
+    _check(lib().nq_conv_implicit_gemm_nested_q8(_ptr(X), _ptr(packed_high), _ptr(packed_low), n_bits, h_bits,
+                                                 ctypes.byref(desc), _ptr(w_scale), ctypes.c_float(act_scale), _ptr(bias),
+                                                 ctypes.c_float(out_scale), int(bool(relu)), _ptr(y),
+                                                 ctypes.c_void_p(workspace.data_ptr() + off), _i64(workspace.numel() - off),
+                                                 _stream()), "nq_conv_implicit_gemm_nested_q8")
     return y
 
 

@@ -312,6 +312,16 @@ int nq_conv_implicit_gemm_nested(const int8_t* X, const void* packed_high, const
                        workspace_bytes, stream, nullptr, packed_low);
 }
 
+int nq_conv_implicit_gemm_nested_q8(const int8_t* X, const void* packed_high, const void* packed_low, int n_bits,
+                                    int h_bits, const nq_conv_desc* d, const float* w_scale, float act_scale,
+                                    const float* bias, float out_scale, int relu, int8_t* Yq, void* workspace,
+                                    int64_t workspace_bytes, void* stream) {
+    const nq::OutQuant oq{out_scale, relu};
+    if (!Yq || !packed_low) return NQ_ERR_INVALID_ARG;
+    return conv_common(X, packed_high, 0, 1, n_bits, h_bits, d, w_scale, act_scale, bias, nullptr, Yq, nq::kOutI8, workspace,
+                       workspace_bytes, stream, &oq, packed_low);
+}
+
 int nq_conv_implicit_gemm_q8(const int8_t* X, const void* Wt, int64_t ldw, int part_bit, int n_bits, int h_bits,
                              const nq_conv_desc* d, const float* w_scale, float act_scale, const float* bias,
                              float out_scale, int relu, int8_t* Yq, void* workspace, int64_t workspace_bytes, void* stream) {

@@ -395,6 +395,15 @@ int nq_gemm_nested(const int8_t* X, int64_t ldx, const void* packed_high, const 
                            ld_acc, Y, ldy, y_dtype, stream, nullptr, packed_low);
 }
 
+int nq_gemm_nested_q8(const int8_t* X, int64_t ldx, const void* packed_high, const void* packed_low, int n_bits, int h_bits,
+                      const float* w_scale, float act_scale, const float* bias, float out_scale, int relu, int64_t M,
+                      int64_t N, int64_t K, int8_t* Yq, int64_t ldyq, void* stream) {
+    const nq::OutQuant oq{out_scale, relu};
+    if (!Yq || !packed_low) return NQ_ERR_INVALID_ARG;
+    return nq::gemm_common(X, ldx, packed_high, 0, true, n_bits, h_bits, w_scale, act_scale, bias, M, N, K, nullptr, 0, Yq,
+                           ldyq, nq::kOutI8, stream, &oq, packed_low);
+}
+
 int nq_gemm_part(const int8_t* X, int64_t ldx, const void* packed_high, int n_bits, int h_bits, const float* w_scale,
                  float act_scale, const float* bias, int64_t M, int64_t N, int64_t K, int32_t* acc_out, int64_t ld_acc,
                  void* Y, int64_t ldy, int y_dtype, void* stream) {

@@ -43,6 +43,10 @@ def test_gemm_both_modes(M, N, K, relu, with_bias):
     got = nq.nq_gemm_part_q8(Xd, hi, N, n, h, wsd, sa, out_scale, relu=relu, bias=bd).cpu().numpy()
     ref = oracle.requant(oracle.gemm_acc(X, wh), ws, sa, n - h, out_scale, bias=bias, relu=relu)
     assert np.array_equal(got, ref)
+    # nested full-bit mode: the full-bit result from the two packed parts
+    got = nq.nq_gemm_nested_q8(Xd, hi, lo, N, n, h, wsd, sa, out_scale, relu=relu, bias=bd).cpu().numpy()
+    ref = oracle.requant(oracle.gemm_acc(X, oracle.recompose(wh, wlo, n, h)), ws, sa, 0, out_scale, bias=bias, relu=relu)
+    assert np.array_equal(got, ref)
     nq.nq_device_status()
 
 
@@ -59,7 +63,7 @@ def test_convolution_both_modes(L):
     ldw = -(-L.K // 16) * 16
     w_mat = dev(wl.oihw_to_ohwi_matrix(W, ldw))[:, :L.K]
     m_mat = dev(wl.oihw_to_ohwi_matrix(mask, ldw))[:, :L.K]
-    hi, _ = nq.nq_decompose(w_mat, m_mat, n, h, True)
+    hi, lo = nq.nq_decompose(w_mat, m_mat, n, h, True)
     desc = nq.nq_conv_desc(batch, L.Cin, L.H, L.W, L.Cout, L.R, L.S, L.stride, L.pad, 1)
     out_scale = 0.9
     for part in (False, True):
@@ -68,6 +72,10 @@ def test_convolution_both_modes(L):
         got = nq.nq_conv_implicit_gemm_q8(dev(X), hi if part else w_mat, desc, dev(ws), sa, out_scale, relu=True,
                                           part_bit=part, n_bits=n, h_bits=h).cpu().numpy()
         assert np.array_equal(got, ref), (L.name, part)
+    ref = oracle.requant(oracle.conv_acc(X, W, L.stride, L.pad).transpose(0, 2, 3, 1), ws, sa, 0, out_scale, relu=True)
+    got = nq.nq_conv_implicit_gemm_nested_q8(dev(X), hi, lo, desc, dev(ws), sa, out_scale, relu=True, n_bits=n,
+                                             h_bits=h).cpu().numpy()
+    assert np.array_equal(got, ref), (L.name, "nested")
     nq.nq_device_status()
 
 
