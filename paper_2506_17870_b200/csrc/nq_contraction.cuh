@@ -434,6 +434,10 @@ __device__ __forceinline__ void store_chunk(const ContractionArgs& p, long long 
 // `row` / `row_ok` its row index and validity; all 32 lanes must call.
 __device__ __forceinline__ void store_rows64(uint8_t* stage, int lane, const uint4 (&q)[4], int row, bool row_ok,
                                              uint8_t* base, long long pitch_bytes, long long col_byte) {
+    // a tile store of the other output may still be reading this block (accumulators by ordinary stores next to a
+    // Y written by tile stores, or the reverse): wait for it before overwriting what it reads
+    if (lane == 0) sm100::bulk_wait_read_all();
+    __syncwarp();
     uint4* mine = reinterpret_cast<uint4*>(stage + lane * kEpiRowPitch);
     mine[0] = q[0]; mine[1] = q[1]; mine[2] = q[2]; mine[3] = q[3];
     __syncwarp();

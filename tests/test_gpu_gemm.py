@@ -214,3 +214,26 @@ def test_rejected_arguments():
     assert e.value.status == 3
     acc, y = nq.nq_gemm_full(X[:0], W, ws, 1.0)  # empty M: nothing to do
     assert y.shape == (0, 64)
+
+
+@pytest.mark.parametrize("acc_plain", [True, False])
+def test_one_output_by_tile_stores_the_other_by_ordinary_stores(acc_plain):
+    """The two outputs of a launch share a warp's staging block.  With one of them on tile stores (aligned) and the
+    other on ordinary stores (pitch not a multiple of 16 bytes) the ordinary path must not overwrite a block that a
+    tile store in flight still reads: many chunks per warp, several launches, every value checked."""
+    M, N, K = 1030, 1100, 256
+    d = wl.gemm_inputs(90, int(acc_plain), M, N, K)
+    Xd, Wd, wsd = dev_padded(d["X"]), dev_padded(d["W"]), dev(d["w_scale"])
+    acc_ref = oracle.gemm_acc(d["X"], d["W"])
+    y_ref = oracle.dequant(acc_ref, d["w_scale"], d["act_scale"], 0)
+    for _ in range(4):
+        if acc_plain:
+            acc = torch.zeros((M, N + 1), dtype=torch.int32, device="cuda")[:, :N]
+            y = torch.full((M, N), float("nan"), dtype=torch.float32, device="cuda")
+        else:
+            acc = torch.zeros((M, N), dtype=torch.int32, device="cuda")
+            y = torch.full((M, N + 1), float("nan"), dtype=torch.float32, device="cuda")[:, :N]
+        nq.nq_gemm_full(Xd, Wd, wsd, d["act_scale"], acc_out=acc, y_out=y)
+        nq.nq_device_status()
+        assert np.array_equal(host(acc), acc_ref)
+        assert np.array_equal(host(y), y_ref)
