@@ -49,8 +49,8 @@ CONV_H = 6
 # a gigabyte per launch): it is taken as four times 8192, every operand and the output growing fourfold.  Must be set
 # to None again when the contraction kernels change.
 NCU_GEMM_DRAM_MB = {
-    4096: {4: 25.6, 5: 27.8, 6: 29.9, 7: 32.3, 0: 34.2},
-    8192: {4: 276.0, 5: 288.0, 6: 313.0, 7: 343.0, 0: 360.0},
+    4096: {4: 25.7, 5: 27.8, 6: 30.0, 7: 32.2, 0: 34.3},
+    8192: {4: 290.0, 5: 287.0, 6: 312.0, 7: 342.0, 0: 358.0},
 }
 
 
