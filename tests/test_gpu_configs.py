@@ -60,8 +60,20 @@ def test_config3_whole_model_page_out_and_page_in_in_one_call():
         assert np.array_equal(host(tensors[i]["packed_low"]), oracle.pack_sliced(wlo, n - h + 1))
 
 
-@pytest.mark.parametrize("name,h", [("l1b0c2", 6), ("l1b0c3", 6), ("l3b1c1", 6), ("l4b0c2", 6),
-                                    ("l3b1c1", 4), ("l4b0c2", 4), ("l1b0c3", 3)])
+def _distinct_resnet101_shapes():
+    """The first layer of every distinct (Cin, H, W, Cout, R, S, stride, pad) of the stack: 24 shapes, the
+    7 x 7 stem (explicit patch matrix) and the classifier included."""
+    seen, names = set(), []
+    for L in wl.resnet101_layers():
+        key = (L.Cin, L.H, L.W, L.Cout, L.R, L.S, L.stride, L.pad)
+        if key not in seen:
+            seen.add(key)
+            names.append(L.name)
+    return names
+
+
+@pytest.mark.parametrize("name,h", [(n, 6) for n in _distinct_resnet101_shapes()] +
+                         [("l3b1c1", 4), ("l4b0c2", 4), ("l1b0c3", 3)])
 def test_config3_convolution_layers_at_batch_128_sampled_pixels(name, h):
     L = next(l for l in wl.resnet101_layers() if l.name == name)
     batch = 128
