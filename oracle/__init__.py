@@ -208,6 +208,47 @@ def requant(acc, w_scale, act_scale: float, l_shift: int, out_scale: float, bias
     return q.reshape(*lead, N)
 
 
+def requant_res(acc, w_scale, act_scale: float, l_shift: int, out_scale: float, res, res_scale: float, bias=None,
+                relu: bool = True):
+    """requant with a residual connection: the INT8 skip tensor `res` (same shape as acc, scale res_scale) is added,
+    dequantised, before the activation (the library's own definition, fp32)."""
+    acc = _c(acc, np.int32)
+    lead = acc.shape[:-1]
+    N = acc.shape[-1]
+    acc2 = acc.reshape(-1, N)
+    M = acc2.shape[0]
+    r = _c(res, np.int8).reshape(-1, N)
+    assert r.shape == acc2.shape
+    ws = _c(w_scale, np.float32)
+    assert ws.shape == (N,)
+    b = None if bias is None else _c(bias, np.float32)
+    q = np.empty((M, N), dtype=np.int8)
+    _load().nqo_requant_res(_p(acc2), _i64(N), _i64(M), _i64(N), _p(ws), ctypes.c_float(act_scale), int(l_shift),
+                            None if b is None else _p(b), _p(r), _i64(N), ctypes.c_float(res_scale), int(bool(relu)),
+                            ctypes.c_float(out_scale), _p(q), _i64(N))
+    return q.reshape(*lead, N)
+
+
+def maxpool_nhwc(x, ksize: int, stride: int, pad: int):
+    """Integer max pooling of INT8 NHWC activations; padding never wins."""
+    x = _c(x, np.int8)
+    B, H, W, C = x.shape
+    Ho, Wo = (H + 2 * pad - ksize) // stride + 1, (W + 2 * pad - ksize) // stride + 1
+    y = np.empty((B, Ho, Wo, C), dtype=np.int8)
+    _load().nqo_maxpool_nhwc(_p(x), _i64(B), _i64(H), _i64(W), _i64(C), _i64(ksize), _i64(stride), _i64(pad), _p(y))
+    return y
+
+
+def avgpool_requant_nhwc(x, in_scale: float, out_scale: float):
+    """Global average pooling of INT8 NHWC activations, requantised to INT8 [B, C]."""
+    x = _c(x, np.int8)
+    B, H, W, C = x.shape
+    y = np.empty((B, C), dtype=np.int8)
+    _load().nqo_avgpool_requant_nhwc(_p(x), _i64(B), _i64(H), _i64(W), _i64(C), ctypes.c_float(in_scale),
+                                     ctypes.c_float(out_scale), _p(y))
+    return y
+
+
 def f32_to_bf16_bits(x):
     x = _c(x, np.float32)
     out = np.empty(x.shape, dtype=np.uint16)

@@ -367,6 +367,95 @@ void nqo_requant(const int32_t *acc, int64_t ldacc, int64_t M, int64_t N,
         }
 }
 
+/* ------------------------------------------------------------------------- */
+/* O6c  the same hand-over with a residual connection (the skip path of a      */
+/*      ResNet block): the skip tensor r is INT8 with its own scale and is     */
+/*      added, dequantised, before the activation.  PARITY UNPINNED by the     */
+/*      paper (it says "8-bit activations" and nothing about the blocks'       */
+/*      arithmetic); the library's own definition, fp32, one rounding each:    */
+/*        v = dequantised output as in O6 (+ bias)                             */
+/*        v = fl(v + fl(float(r) * res_scale))                                 */
+/*        v = max(v, 0) when relu;  t = fl(v * fl(1 / out_scale))              */
+/*        q = clip(round-half-even(t), -128, 127)                              */
+/* ------------------------------------------------------------------------- */
+void nqo_requant_res(const int32_t *acc, int64_t ldacc, int64_t M, int64_t N,
+                     const float *w_scale, float act_scale, int l_shift, const float *bias,
+                     const int8_t *res, int64_t ldres, float res_scale,
+                     int relu, float out_scale, int8_t *q, int64_t ldq)
+{
+    const float pow2 = (float)(1 << l_shift);
+    volatile float inv = 1.0f / out_scale;
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t j = 0; j < N; ++j) {
+            volatile float sj = act_scale * w_scale[j];
+            volatile float scale = sj * pow2;
+            volatile float v = (float)acc[m * ldacc + j] * scale;
+            if (bias) { volatile float t = v + bias[j]; v = t; }
+            volatile float skip = (float)res[m * ldres + j] * res_scale;
+            volatile float sum = v + skip;
+            v = sum;
+            if (relu && v < 0.0f) v = 0.0f;
+            volatile float t = v * inv;
+            float r = nearbyintf(t);
+            if (r < -128.0f) r = -128.0f;
+            if (r > 127.0f) r = 127.0f;
+            q[m * ldq + j] = (int8_t)r;
+        }
+}
+
+/* ------------------------------------------------------------------------- */
+/* O8   pooling between the layers of a chained model (library's own           */
+/*      definitions, PARITY UNPINNED by the paper).  Activations are INT8,     */
+/*      NHWC [B, H, W, C].                                                     */
+/*      max pooling: the integer maximum over the window's taps that lie       */
+/*      inside the image (padding never wins); the scale is unchanged.         */
+/*      global average pooling with requantisation:                            */
+/*        sum = integer sum over the H * W pixels of a channel                 */
+/*        a   = fl(in_scale / float(H * W))                                    */
+/*        t   = fl(fl(float(sum) * a) * fl(1 / out_scale))                     */
+/*        q   = clip(round-half-even(t), -128, 127)                            */
+/* ------------------------------------------------------------------------- */
+void nqo_maxpool_nhwc(const int8_t *x, int64_t B, int64_t H, int64_t W, int64_t C,
+                      int64_t ksize, int64_t stride, int64_t pad, int8_t *y)
+{
+    const int64_t Ho = (H + 2 * pad - ksize) / stride + 1, Wo = (W + 2 * pad - ksize) / stride + 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t b = 0; b < B; ++b)
+        for (int64_t p = 0; p < Ho; ++p)
+            for (int64_t q = 0; q < Wo; ++q)
+                for (int64_t c = 0; c < C; ++c) {
+                    int best = -128;
+                    for (int64_t r = 0; r < ksize; ++r)
+                        for (int64_t s = 0; s < ksize; ++s) {
+                            int64_t ih = p * stride - pad + r, iw = q * stride - pad + s;
+                            if (ih < 0 || ih >= H || iw < 0 || iw >= W) continue;
+                            int v = x[((b * H + ih) * W + iw) * C + c];
+                            if (v > best) best = v;
+                        }
+                    y[((b * Ho + p) * Wo + q) * C + c] = (int8_t)best;
+                }
+}
+
+void nqo_avgpool_requant_nhwc(const int8_t *x, int64_t B, int64_t H, int64_t W, int64_t C,
+                              float in_scale, float out_scale, int8_t *y)
+{
+    volatile float a = in_scale / (float)(H * W);
+    volatile float inv = 1.0f / out_scale;
+#pragma omp parallel for schedule(static)
+    for (int64_t b = 0; b < B; ++b)
+        for (int64_t c = 0; c < C; ++c) {
+            int32_t sum = 0;
+            for (int64_t i = 0; i < H * W; ++i) sum += x[(b * H * W + i) * C + c];
+            volatile float v = (float)sum * a;
+            volatile float t = v * inv;
+            float r = nearbyintf(t);
+            if (r < -128.0f) r = -128.0f;
+            if (r > 127.0f) r = 127.0f;
+            y[b * C + c] = (int8_t)r;
+        }
+}
+
 /* fp32 -> bf16, round to nearest, ties to even (finite inputs) */
 void nqo_f32_to_bf16(const float *x, int64_t count, uint16_t *out)
 {

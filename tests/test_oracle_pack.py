@@ -2,8 +2,8 @@
 
 The paper fixes only the field content (k-bit two's complement, e.g. 1011 for -5 and 01101 for 13)
 and, for its packed-bit tensor, 64 // k fields per unsigned 64-bit word.  The bit positions of the
-sliced layout are this library's own; they are pinned by a hand-laid example written out below from
-the layout's prose definition, by the size function and by round trips.
+sliced layout are this library's own; they are pinned by literal bytes worked out by hand from the
+layout's prose definition (field widths 3, 4, 5, 6, 7 and 8), by the size function and by round trips.
 """
 import numpy as np
 import pytest
@@ -52,33 +52,6 @@ def test_sliced_padding_is_zero_and_size_is_k_over_8_bytes_per_weight():
     assert oracle.sliced_row_bytes(128 * 64, 5) * 8 == 128 * 64 * 5
 
 
-def _lay_by_hand(values, bits):
-    """The sliced layout written out again, straight from its prose definition, bit by bit."""
-    widths = [s for s in (8, 4, 2, 1) if bits & s]
-    out = np.zeros(16 * bits, dtype=np.uint8)
-    for e, val in enumerate(values):
-        field = int(val) & ((1 << bits) - 1)
-        text = format(field, f"0{bits}b")            # most significant bit first
-        base, used = 0, 0
-        for s in widths:
-            piece = int(text[used:used + s], 2)
-            unit, quad, lane = e // 32, (e % 32) // 4, e % 4
-            per_byte = 8 // s
-            word, sub = quad // per_byte, quad % per_byte
-            byte = base + (unit * s + word) * 4 + lane
-            out[byte] |= piece << (8 - s * (sub + 1))
-            base += 16 * s
-            used += s
-    return out
-
-
-@pytest.mark.parametrize("bits", range(1, 9))
-def test_sliced_layout_against_a_hand_laid_group(bits):
-    rng = np.random.default_rng(99 + bits)
-    v = rng.integers(-(2 ** (bits - 1)), 2 ** (bits - 1), size=(1, 128)).astype(np.int8)
-    assert np.array_equal(oracle.pack_sliced(v, bits)[0], _lay_by_hand(v[0], bits))
-
-
 def test_sliced_layout_literal_bytes():
     # INT4 fields, element 0 = -5 (1011), element 4 = 7 (0111): they share byte 0 (lane 0 of word 0),
     # element 0 in the top nibble.  Element 1 = 3 goes to byte 1's top nibble.  Element 32 opens unit 1.
@@ -95,3 +68,53 @@ def test_sliced_layout_literal_bytes():
     # INT8 is the plain byte order
     v8 = np.arange(-64, 64, dtype=np.int8)[None, :]
     assert np.array_equal(oracle.pack_sliced(v8, 8)[0].view(np.int8), v8[0])
+
+
+def _packed_group_bytes(bits, placed, cols=128):
+    v = np.zeros((1, cols), dtype=np.int8)
+    for e, val in placed.items():
+        v[0, e] = val
+    return oracle.pack_sliced(v, bits)[0]
+
+
+def test_sliced_layout_literal_bytes_six_bit_fields():
+    """INT(8|6) stores w_high in 6-bit fields: a 4-bit slice (bytes 0..63 of a group) over a 2-bit slice (64..95).
+    Worked out by hand from the layout's prose: element e sits, in the slice of width s, in byte
+    ((e/32)*s + ((e%32)/4) / (8/s)) * 4 + e%4 at bits [8 - s*(sub+1), 8 - s*sub), sub = ((e%32)/4) % (8/s)."""
+    p = _packed_group_bytes(6, {0: -5, 4: 13, 13: -32, 45: 31, 127: -1, 128: 1}, cols=256)
+    assert len(p) == 2 * 96
+    # e = 0: -5 = 111011 -> 1110 | 11;  e = 4: 13 = 001101 -> 0011 | 01 (same byte lane, next sub-position)
+    assert p[0] == 0xE3 and p[64] == 0xD0
+    # e = 13: -32 = 100000 -> 1000 | 00: word 1, lane 1, low nibble; nothing in the 2-bit slice
+    assert p[5] == 0x08
+    # e = 45 (unit 1, element 13 of it): 31 = 011111 -> 0111 | 11
+    assert p[21] == 0x07 and p[73] == 0x03
+    # e = 127, the group's last element: -1 = 111111
+    assert p[63] == 0x0F and p[95] == 0x03
+    # e = 128 opens the second group, 96 bytes on: 1 = 000001 -> 0000 | 01 in the top two bits
+    assert p[96] == 0x00 and p[160] == 0x40
+    assert np.count_nonzero(p) == 8
+
+
+def test_sliced_layout_literal_bytes_three_bit_fields():
+    """INT(8|6) stores the compensated w_low in 3-bit fields: a 2-bit slice (bytes 0..31) over a 1-bit slice (32..47)."""
+    p = _packed_group_bytes(3, {0: -3, 8: 3, 30: -4, 81: 2, 127: -1})
+    assert len(p) == 48
+    # e = 0: -3 = 101 -> 10 | 1;  e = 8: 3 = 011 -> 01 | 1 (same lane, third sub-position of both slices)
+    assert p[0] == 0x84 and p[32] == 0xA0
+    # e = 30 (quad 7, lane 2): -4 = 100 -> 10 | 0: word 1 of the 2-bit slice, last sub-position
+    assert p[6] == 0x02
+    # e = 81 (unit 2, element 17: quad 4, lane 1): 2 = 010 -> 01 | 0
+    assert p[21] == 0x40
+    # e = 127: -1 = 111
+    assert p[31] == 0x03 and p[47] == 0x01
+    assert np.count_nonzero(p) == 6
+
+
+def test_sliced_layout_literal_bytes_seven_bit_fields():
+    """Three slices: 4 bits (bytes 0..63), 2 bits (64..95), 1 bit (96..111)."""
+    p = _packed_group_bytes(7, {5: -64, 6: 63})
+    assert len(p) == 112
+    # e = 5 (quad 1, lane 1): -64 = 1000000 -> 1000 | 00 | 0;  e = 6 (quad 1, lane 2): 63 = 0111111 -> 0111 | 11 | 1
+    assert p[1] == 0x08 and p[2] == 0x07 and p[66] == 0x30 and p[98] == 0x40
+    assert np.count_nonzero(p) == 4
