@@ -7,7 +7,9 @@ One "step" is one pass of the whole path over the large square GEMM sweep (M = N
     decompose -> drop-low (page-out) -> recompose (page-in) -> part-bit GEMM,   plus one full-bit GEMM per size,
 
 followed by the ResNet-18-shaped convolution stack (config 2: 20 convolutions + classifier, batch 32, NCHW
-int8 activations, implicit GEMM, both modes).  After the timed steps the whole-model page-out / page-in of a
+int8 activations, implicit GEMM, both modes; each mode's stack is replayed as one CUDA graph).  Before the warm-up
+the INT8 tensor ceiling is measured (nq_i8_mma_ceiling: the GEMMs' tensor instruction issued from shared memory with
+no loads, burst and sustained): roofline.frac is the GEMM launches' rate over the sustained ceiling.  After the timed steps the whole-model page-out / page-in of a
 ResNet-101-shaped and a ViT-B-shaped model (one batched launch each, cold L2) is timed separately and
 reported under rows.model_switch, and configs 3 and 5 run layer by layer through both modes (the ResNet-101-shaped
 stack at batch 128, the ViT-B/16 linears at 256 x 197 tokens): rows.resnet101_stack_int8_6, rows.vit_b16_linears_int8_4.
@@ -44,31 +46,27 @@ METRIC = "nested_int8_gemm_tops"
 CONV_H = 6
 
 
-# DRAM bytes (read + written, MB) of one GEMM launch, from the ncu capture summarised in
-# profiles/gemm_dram_traffic_4096_8192.md (tile-store epilogue, 40 ns barrier probes, packed-tile producer warp).  16384 was not captured (over
-# a gigabyte per launch): it is taken as four times 8192, every operand and the output growing fourfold.  Must be set
-# to None again when the contraction kernels change.
-NCU_GEMM_DRAM_MB = {
-    4096: {4: 25.7, 5: 27.8, 6: 30.0, 7: 32.2, 0: 34.3},
-    8192: {4: 290.0, 5: 287.0, 6: 312.0, 7: 342.0, 0: 358.0},
-}
+# DRAM traffic of the GEMM launches comes from an ncu capture, never from this file: profiles/gemm_dram_traffic.txt is
+# written by `python -m paper_2506_17870_b200.ncu_traffic` from the capture's CSV and carries a hash of the kernel
+# sources it was taken on.  When the sources have changed since, or a size was not captured, traffic is null.
+TRAFFIC_FILE = ROOT / "profiles" / "gemm_dram_traffic.txt"
 
 
 def gemm_traffic_bytes_per_launch(sizes):
-    """Mean DRAM traffic of the GEMM launches of one step (h = 4..7 part-bit + one full-bit per size), or None."""
-    if NCU_GEMM_DRAM_MB is None:
-        return None
-    total, n = 0.0, 0
-    for s in sizes:
-        table, factor = NCU_GEMM_DRAM_MB.get(s), 1.0
-        if table is None and s == 16384:
-            table, factor = NCU_GEMM_DRAM_MB.get(8192), 4.0
-        if table is None:
-            return None
-        for h in list(HS) + [0]:
-            total += table[h] * factor * 1e6
-            n += 1
-    return total / n
+    """(mean DRAM bytes of the GEMM launches of one step, note).  The mean runs over the captured sizes among
+    `sizes` (h = 4..7 part-bit + one full-bit launch each); None with the reason when there is nothing valid."""
+    from paper_2506_17870_b200 import ncu_traffic
+    table, why = ncu_traffic.load(TRAFFIC_FILE)
+    if table is None:
+        return None, why
+    have = [s for s in sizes if all((s, h) in table for h in list(HS) + [0])]
+    if not have:
+        return None, "no size of this run was captured"
+    vals = [table[(s, h)] for s in have for h in list(HS) + [0]]
+    note = "ncu dram__bytes_read + dram__bytes_write, mean over the GEMM launches of sizes %s" % ",".join(map(str, have))
+    if len(have) < len(sizes):
+        note += " only (%s not captured: over a gigabyte per launch)" % ",".join(str(s) for s in sizes if s not in have)
+    return float(np.mean(vals)), note
 
 
 def measured_peaks():
@@ -204,6 +202,53 @@ def whole_job_tops(world, ops_per_gpu_per_step, ms_per_step):
     return world * ops_per_gpu_per_step / (ms_per_step * 1e-3) / 1e12
 
 
+# --------------------------------------------------------------------------- measured INT8 tensor ceiling
+def measure_int8_ceiling(nq, torch, gpu_index, seconds=2.0):
+    """The issue-only rate of the tensor instruction the GEMMs use (nq_i8_mma_ceiling: tcgen05.mma kind::i8 on CTA
+    pairs, operands parked in shared memory, accumulators in tensor memory, no loads, no epilogue), in TOP/s.
+    burst      best of five 1 ms launches after the GPU has idled for half a second (a kernel timed alone)
+    sustained  median over the second half of about `seconds` of back-to-back 10 ms launches (a kernel inside a
+               long hot step: the 1 kW power limit has pulled the clock down by then)
+    with the median SM clock sampled during the sustained run."""
+    stream = torch.cuda.current_stream()
+
+    def launch(iters):
+        a = torch.cuda.Event(enable_timing=True)
+        b = torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        ops = nq.nq_i8_mma_ceiling(iters)
+        b.record(stream)
+        return a, b, ops
+
+    launch(400)
+    torch.cuda.synchronize()
+    nq.nq_device_status()
+    time.sleep(0.5)
+    burst = 0.0
+    for _ in range(5):
+        a, b, ops = launch(3700)
+        torch.cuda.synchronize()
+        burst = max(burst, ops / (a.elapsed_time(b) * 1e-3) / 1e12)
+    sampler = ClockSampler(gpu_index)
+    sampler.start()
+    time.sleep(0.2)
+    t0 = time.time()
+    evs = []
+    while time.time() - t0 < seconds and len(evs) < 400:
+        for _ in range(8):
+            evs.append(launch(37000))
+        evs[-1][1].synchronize()
+    torch.cuda.synchronize()
+    t1 = time.time()
+    clocks = sampler.stop(t0 + 0.5 * (t1 - t0), t1)
+    rates = [ops / (a.elapsed_time(b) * 1e-3) / 1e12 for a, b, ops in evs[len(evs) // 2:]]
+    nq.nq_device_status()
+    return {"burst_tops": round(burst, 1), "sustained_tops": round(float(np.median(rates)), 1),
+            "sustained_sm_mhz": clocks.get("sm_mhz"), "sustained_reasons": clocks.get("reasons"),
+            "launches": len(evs), "how": "nq_i8_mma_ceiling: 74 CTA pairs issuing tcgen05.mma.cta_group::2.kind::i8 "
+                                         "256x256x32 from shared memory into tensor memory, no loads"}
+
+
 # --------------------------------------------------------------------------- our arm
 def run_ours(args, rank, world, local_rank):
     import torch
@@ -235,6 +280,13 @@ def run_ours(args, rank, world, local_rank):
         conv_layers = conv_bench_layers()
         conv_state = [_prepare_conv(nq, wl, torch, L, args.conv_batch, i, dev) for i, L in enumerate(conv_layers)]
 
+    conv_graphs = {}
+    if have_conv and args.graphs:
+        for part in (False, True):
+            g = capture_stack(torch, conv_state, lambda cs: _run_conv(nq, cs, part))
+            if g is not None:
+                conv_graphs[part] = g
+
     launches = [0]
     events = {}
 
@@ -259,11 +311,18 @@ def run_ours(args, rank, world, local_rank):
                 timed(("page_in", s, h), lambda: nq.nq_recompose(d["hi"][h], d["lo"][h], s, s, N_BITS, h, True, out=d["w_rec"]), record)
                 timed(("gemm_part", s, h), lambda: nq.nq_gemm_part(d["X"], d["hi"][h], s, N_BITS, h, d["w_scale"], ACT_SCALE, y_out=d["y"]), record)
             timed(("gemm_full", s, 0), lambda: nq.nq_gemm_full(d["X"], d["w_rec"], d["w_scale"], ACT_SCALE, y_out=d["y"]), record)
-        for L, cs in zip(conv_layers, conv_state):
-            timed(("conv_full", L.name, 0), lambda: _run_conv(nq, cs, False), record, 2)   # layout pre-pass + contraction
-            timed(("conv_part", L.name, 0), lambda: _run_conv(nq, cs, True), record, 2)
+        # config 2: each stack is one CUDA-graph launch (layout pre-pass + contraction of every layer, in order) when
+        # the capture succeeded, otherwise layer by layer
+        if len(conv_graphs) == 2:
+            timed(("conv_stack_graph", "full_bit", 0), lambda: conv_graphs[False].replay(), record, 2 * len(conv_layers))
+            timed(("conv_stack_graph", "part_bit", 0), lambda: conv_graphs[True].replay(), record, 2 * len(conv_layers))
+        else:
+            for L, cs in zip(conv_layers, conv_state):
+                timed(("conv_full", L.name, 0), lambda: _run_conv(nq, cs, False), record, 2)   # layout pre-pass + contraction
+                timed(("conv_part", L.name, 0), lambda: _run_conv(nq, cs, True), record, 2)
 
-    ops_step = sum(2.0 * s ** 3 * (len(HS) + 1) for s in sizes)
+    ops_gemm_sweep = sum(2.0 * s ** 3 * (len(HS) + 1) for s in sizes)
+    ops_step = ops_gemm_sweep
     for L in conv_layers:
         M, N, K = L.gemm_view(args.conv_batch)
         ops_step += 2 * 2.0 * M * N * K
@@ -273,6 +332,10 @@ def run_ours(args, rank, world, local_rank):
             torch.distributed.barrier()
         torch.cuda.synchronize()
 
+    ceiling = measure_int8_ceiling(nq, torch, local_rank) if args.ceiling else None
+    peaks = measured_peaks()
+    peaks["int8_tops"] = ceiling["sustained_tops"] if ceiling else 2.0 * peaks["bf16_tflops_sustained"]
+    peaks["int8_source"] = "measured ceiling (sustained)" if ceiling else "2 x bf16 sustained"
     for _ in range(args.warmup):
         step(False)
     barrier()
@@ -299,7 +362,7 @@ def run_ours(args, rank, world, local_rank):
 
     e2e = _run_e2e(nq, torch, sizes, host, state, args, world)
     model_switch = _model_switch(nq, torch, wl, dev) if (rank == 0 and args.model_switch) else None
-    model_rows = _model_rows(nq, torch, wl, dev, args.model_batch) if (rank == 0 and args.model_rows and have_conv) else None
+    model_rows = _model_rows(nq, torch, wl, dev, args.model_batch, peaks) if (rank == 0 and args.model_rows and have_conv) else None
 
     total_ms, e2e["ms_per_step"] = max_over_ranks([total_ms, e2e["ms_per_step"]], world, dev)
     ms_per_step = total_ms / args.steps
@@ -307,8 +370,9 @@ def run_ours(args, rank, world, local_rank):
     if rank != 0:
         return None
 
-    peaks = measured_peaks()
     rows = _summarise_rows(events, conv_layers, args.conv_batch, peaks)
+    if have_conv:
+        rows.update(_config2_rows(nq, torch, wl, conv_layers, conv_state, args.conv_batch, peaks, events))
     gemm_ms, gemm_ops, gemm_n = 0.0, 0.0, 0
     for (kind, s, h), pairs in events.items():
         if kind in ("gemm_full", "gemm_part"):
@@ -316,20 +380,32 @@ def run_ours(args, rank, world, local_rank):
                 gemm_ms += a.elapsed_time(b)
                 gemm_ops += 2.0 * s ** 3
                 gemm_n += 1
-    int8_peak = 2.0 * peaks["bf16_tflops"]
+    # Denominator: the measured ceiling of the INT8 tensor instruction on this GPU (sustained: these launches run
+    # inside a long hot step).  Alongside: its burst figure, 2 x the measured bf16 cuBLAS figures (dense INT8 :
+    # bf16 nominal ratio 4.5 : 2.25) and the nominal 4.5 POP/s.
+    derived_burst, derived_sustained = 2.0 * peaks["bf16_tflops"], 2.0 * peaks["bf16_tflops_sustained"]
     achieved = gemm_ops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
+    if ceiling is not None:
+        int8_peak, peak_source = ceiling["sustained_tops"], "measured in this run: sustained issue-only rate of tcgen05.mma kind::i8 (nq_i8_mma_ceiling)"
+    else:
+        int8_peak, peak_source = derived_sustained, "derived: 2 x the %s bf16 sustained figure" % peaks["source"]
+    traffic, traffic_note = gemm_traffic_bytes_per_launch(sizes)
     roofline = {
         "bound": "tensor", "kernel": "contraction_pair_kernel / contraction_kernel (tcgen05 kind::i8): every GEMM launch of the timed steps",
         "achieved": round(achieved, 1), "peak": round(int8_peak, 1), "unit": "TOP/s",
-        "frac": round(achieved / int8_peak, 4),
-        "peak_source": "2 x the %s bf16 burst figure (dense INT8 : bf16 nominal ratio 4.5 : 2.25)" % peaks["source"],
+        "frac": round(achieved / int8_peak, 4), "peak_source": peak_source,
+        "int8_ceiling": ceiling,
+        "frac_vs_measured_burst": round(achieved / ceiling["burst_tops"], 4) if ceiling else None,
+        "frac_vs_2x_bf16_burst": round(achieved / derived_burst, 4),
+        "frac_vs_2x_bf16_sustained": round(achieved / derived_sustained, 4),
+        "frac_vs_nominal_4500": round(achieved / 4500.0, 4),
         "launches": gemm_n, "avg_launch_ms": round(gemm_ms / max(gemm_n, 1), 4),
-        "traffic": gemm_traffic_bytes_per_launch(sizes),
-        "traffic_unit": "DRAM bytes per launch, mean over the step's GEMM launches (ncu, profiles/gemm_dram_traffic_4096_8192.md)",
+        "traffic": traffic, "traffic_note": traffic_note,
         "algorithmic_bytes_per_launch": float(np.mean([s * s * (1 + (h / 8.0 if h else 1.0) + 2) for s in sizes for h in list(HS) + [0]])),
     }
-    conv_note = (", + config 2: the ResNet-18-shaped stack (%d layers), batch %d, NCHW int8 in, both modes"
-                 % (len(conv_layers), args.conv_batch) if have_conv else "")
+    conv_note = (", + config 2: the ResNet-18-shaped stack (%d layers), batch %d, NCHW int8 in, both modes%s"
+                 % (len(conv_layers), args.conv_batch, ", each stack one CUDA-graph launch" if len(conv_graphs) == 2 else "")
+                 if have_conv else "")
     line = {
         "metric": METRIC, "value": round(value, 2), "unit": "TOPS", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak",
@@ -341,15 +417,17 @@ def run_ours(args, rank, world, local_rank):
                                            "between two launches of the same kernel)",
                    "per_gpu_ops_per_step": ops_step},
         "clocks": clocks, "gpu_launches": gpu_launches,
-        "e2e": {"value": round(whole_job_tops(world, ops_step, e2e["ms_per_step"]), 3), "unit": "TOPS",
+        "e2e": {"value": round(whole_job_tops(world, ops_gemm_sweep, e2e["ms_per_step"]), 3), "unit": "TOPS",
                 "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
-                "ms_per_step": round(e2e["ms_per_step"], 3), "covers": "the GEMM sweep (codec + both GEMM modes)"},
+                "ms_per_step": round(e2e["ms_per_step"], 3), "ops_per_step": ops_gemm_sweep,
+                "covers": "the GEMM sweep (codec + both GEMM modes), whose ops alone are counted; no convolution stack"},
         "roofline": roofline, "rows": rows,
     }
     if model_switch is not None:
         line["rows"]["model_switch"] = model_switch
         line["rows"]["word64_convert_8192"] = _word64_rows(nq, torch, dev)
-        line["rows"]["gemm_nested_8192"] = _nested_rows(nq, torch, dev)
+        line["rows"]["gemm_nested_8192"] = _nested_rows(nq, torch, dev, peaks)
+        line["rows"]["gemm_output_types_config4"] = _output_type_rows(nq, torch, state, sizes, peaks)
     if model_rows is not None:
         line["rows"].update(model_rows)
     if world == 1 and not args.no_cpu_baseline:
@@ -357,9 +435,27 @@ def run_ours(args, rank, world, local_rank):
     return line
 
 
+def layer_roofline_us(M, N, K, in_bytes, weight_bytes, out_bytes, peaks):
+    """Lower bound of one layer's time: max(integer ops / INT8 tensor ceiling, algorithmic bytes / HBM copy bandwidth),
+    the activations read once, the weights once, the output written once."""
+    t_ops = 2.0 * M * N * K / (peaks["int8_tops"] * 1e12)
+    t_mem = (in_bytes + weight_bytes + out_bytes) / (peaks["hbm_gbs"] * 1e9)
+    return 1e6 * max(t_ops, t_mem)
+
+
+def conv_roofline_us(L, batch, part, h, out_esize, peaks):
+    M, N, K = L.gemm_view(batch)
+    return layer_roofline_us(M, N, K, batch * L.Cin * L.H * L.W, N * K * (h / 8.0 if part else 1.0), M * N * out_esize, peaks)
+
+
+def _frac(t, peaks):
+    return {"frac_int8_ceiling": round(t / peaks["int8_tops"], 3),
+            "frac_2x_bf16_burst": round(t / (2.0 * peaks["bf16_tflops"]), 3),
+            "frac_nominal_4500": round(t / 4500.0, 3)}
+
+
 def _summarise_rows(events, conv_layers, conv_batch, peaks):
     out = {"gemm_full": {}, "gemm_part": {}, "codec": {}}
-    int8_peak = 2.0 * peaks["bf16_tflops"]
     hbm = peaks["hbm_gbs"]
     codec_bytes = {"decompose": 1 + 1 + 9 / 8, "page_out": 1 + 9 / 8, "page_in": 9 / 8 + 1}   # per weight, n = 8
     agg = {}
@@ -367,29 +463,86 @@ def _summarise_rows(events, conv_layers, conv_batch, peaks):
         ms = float(np.mean([a.elapsed_time(b) for a, b in pairs]))
         if kind == "gemm_full":
             t = 2.0 * s ** 3 / (ms * 1e-3) / 1e12
-            out["gemm_full"][str(s)] = {"tops": round(t, 1), "frac_int8_peak": round(t / int8_peak, 3), "ms": round(ms, 4)}
+            out["gemm_full"][str(s)] = {"tops": round(t, 1), "ms": round(ms, 4), **_frac(t, peaks)}
         elif kind == "gemm_part":
             t = 2.0 * s ** 3 / (ms * 1e-3) / 1e12
-            out["gemm_part"].setdefault(str(s), {})[f"h{h}"] = {"tops": round(t, 1), "frac_int8_peak": round(t / int8_peak, 3),
-                                                                "ms": round(ms, 4)}
+            out["gemm_part"].setdefault(str(s), {})[f"h{h}"] = {"tops": round(t, 1), "ms": round(ms, 4), **_frac(t, peaks)}
         elif kind in codec_bytes:
-            agg.setdefault((kind, s), []).append(codec_bytes[kind] * s * s / (ms * 1e-3) / 1e9)
+            agg.setdefault((kind, s), []).append((codec_bytes[kind] * s * s / (ms * 1e-3) / 1e9, h, ms))
         elif kind in ("conv_full", "conv_part"):
             L = next(l for l in conv_layers if l.name == s)
             M, N, K = L.gemm_view(conv_batch)
             t = 2.0 * M * N * K / (ms * 1e-3) / 1e12
-            out.setdefault(kind, {})[s] = {"tops": round(t, 1), "ms": round(ms, 4), "gemm_view": [M, N, K]}
+            roof = conv_roofline_us(L, conv_batch, kind == "conv_part", CONV_H, 2, peaks)
+            out.setdefault(kind, {})[s] = {"tops": round(t, 1), "ms": round(ms, 4), "gemm_view": [M, N, K],
+                                           "roofline_us": round(roof, 2), "frac_roofline": round(roof / (ms * 1e3), 3)}
     for kind in ("conv_full", "conv_part"):
         if kind in out:
             tot_ms = sum(v["ms"] for v in out[kind].values())
             tot_ops = sum(2.0 * v["gemm_view"][0] * v["gemm_view"][1] * v["gemm_view"][2] for v in out[kind].values())
+            roof = sum(v["roofline_us"] for v in out[kind].values())
             out[kind + "_stack"] = {"ms": round(tot_ms, 4), "tops": round(tot_ops / (tot_ms * 1e-3) / 1e12, 1),
-                                    "layers": len(out[kind])}
+                                    "layers": len(out[kind]), "roofline_sum_us": round(roof, 1),
+                                    "frac_roofline": round(roof / (tot_ms * 1e3), 3),
+                                    "roofline": "per layer max(ops / INT8 ceiling, (activations + weights + bf16 output) / HBM), summed"}
     for (kind, s), vals in agg.items():
-        g = float(np.mean(vals))
-        out["codec"].setdefault(kind, {})[str(s)] = {"gbs": round(g, 0), "frac_hbm": round(g / hbm, 3)}
+        g = float(np.mean([v[0] for v in vals]))
+        row = {"gbs": round(g, 0), "frac_hbm": round(g / hbm, 3)}
+        if kind == "page_in":
+            # the paper's switching-overhead model counts only the bytes paged in, P_low = (l + 1) / 8 per weight
+            row["paper_model_p_low_gbs"] = {f"h{h}": round((N_BITS - h + 1) / 8.0 * s * s / (ms * 1e-3) / 1e9, 0) for _, h, ms in vals}
+        out["codec"].setdefault(kind, {})[str(s)] = row
     out["codec"]["algorithmic_bytes_per_weight"] = codec_bytes
-    out["peaks"] = {"int8_tops": int8_peak, "hbm_gbs": hbm, "source": peaks["source"]}
+    out["peaks"] = {"int8_tops": peaks["int8_tops"], "int8_source": peaks["int8_source"], "hbm_gbs": hbm,
+                    "bf16_tflops": peaks["bf16_tflops"], "source": peaks["source"]}
+    return out
+
+
+def _config2_rows(nq, torch, wl, conv_layers, conv_state, conv_batch, peaks, events):
+    """Config 2 layer by layer (outside the timed steps: own CUDA events per layer, median of 3 passes), each layer
+    against its roofline max(ops / INT8 ceiling, algorithmic bytes / HBM); the stack with NHWC input (no layout
+    pre-pass) and with fp32 output; and the graph launches of the timed steps."""
+    out = {}
+    ops = sum(2.0 * float(np.prod(L.gemm_view(conv_batch))) for L in conv_layers)
+    for part in (False, True):
+        kind = "conv_part" if part else "conv_full"
+        ms_l = time_layers(torch, conv_state, lambda cs: _run_conv(nq, cs, part))
+        rows, roof_sum = {}, 0.0
+        for L, ms in zip(conv_layers, ms_l):
+            M, N, K = L.gemm_view(conv_batch)
+            roof = conv_roofline_us(L, conv_batch, part, CONV_H, 2, peaks)
+            roof_sum += roof
+            rows[L.name] = {"tops": round(2.0 * M * N * K / (float(ms) * 1e-3) / 1e12, 1), "us": round(float(ms) * 1e3, 1),
+                            "gemm_view": [M, N, K], "roofline_us": round(roof, 2), "frac_roofline": round(roof / (float(ms) * 1e3), 3)}
+        out[kind] = rows
+        tot = float(ms_l.sum())
+        stack = {"ms": round(tot, 4), "tops": round(ops / (tot * 1e-3) / 1e12, 1), "layers": len(conv_layers),
+                 "roofline_sum_us": round(roof_sum, 1), "frac_roofline": round(roof_sum / (tot * 1e3), 3),
+                 "roofline": "per layer max(ops / INT8 ceiling, (activations + weights + bf16 output) / HBM), summed"}
+        pairs = events.get(("conv_stack_graph", "part_bit" if part else "full_bit", 0))
+        if pairs:
+            gms = float(np.mean([a.elapsed_time(b) for a, b in pairs]))
+            stack["graph_ms_in_step"] = round(gms, 4)
+            stack["graph_frac_roofline"] = round(roof_sum / (gms * 1e3), 3)
+        out[kind + "_stack"] = stack
+    # the same stack fed NHWC activations (no transposing pre-pass; the stem still builds its patch matrix), and with fp32 output
+    nhwc = []
+    for L, cs in zip(conv_layers, conv_state):
+        c = dict(cs)
+        c["x"] = cs["x"].permute(0, 2, 3, 1).contiguous()
+        c["desc"] = nq.nq_conv_desc(conv_batch, L.Cin, L.H, L.W, L.Cout, L.R, L.S, L.stride, L.pad, 0)
+        c["y32"] = torch.empty(cs["y"].shape, dtype=torch.float32, device=cs["y"].device)
+        nhwc.append(c)
+    for part in (False, True):
+        roof = sum(conv_roofline_us(L, conv_batch, part, CONV_H, 2, peaks) for L in conv_layers)
+        row, _ = stack_row(torch, nhwc, lambda cs: _run_conv(nq, cs, part), ops, roof)
+        out[("conv_part" if part else "conv_full") + "_stack_nhwc_in"] = row
+        base = out[("conv_part" if part else "conv_full") + "_stack"]
+        base["nchw_prepass_ms"] = round(base["ms"] - row["ms"], 4)
+    roof = sum(conv_roofline_us(L, conv_batch, False, CONV_H, 4, peaks) for L in conv_layers)
+    out["conv_full_stack_nhwc_in_fp32_out"], _ = stack_row(
+        torch, nhwc, lambda cs: nq.nq_conv_implicit_gemm(cs["x"], cs["w"], cs["desc"], cs["ws"], cs["act"], part_bit=False,
+                                                         workspace=cs["work"], y_out=cs["y32"]), ops, roof)
     return out
 
 
@@ -436,6 +589,8 @@ def _model_switch(nq, torch, wl, dev):
             ms = float(np.median(ts))
             gbs = nbytes / (ms * 1e-3) / 1e9
             res[kind] = {"us": round(ms * 1e3, 1), "gbs": round(gbs, 0), "frac_hbm": round(gbs / peaks["hbm_gbs"], 3)}
+            if kind == "page_in":       # the paper's switching-overhead model counts only the paged bytes, P_low
+                res[kind]["paper_model_p_low_gbs"] = round(weights * (N_BITS - h + 1) / 8.0 / (ms * 1e-3) / 1e9, 0)
         res["weights"] = weights
         res["tensors"] = len(shapes)
         res["algorithmic_mb"] = round(nbytes / 1e6, 1)
@@ -443,11 +598,9 @@ def _model_switch(nq, torch, wl, dev):
     return out
 
 
-def _nested_rows(nq, torch, dev):
+def _nested_rows(nq, torch, dev, peaks):
     """The full-bit layer computed straight from packed w_high and compensated w_low (no INT8 copy of the weights):
-    8192^3, median of 5 launches per nesting, against the int8 peak; outputs checked equal to the full-bit GEMM's."""
-    peaks = measured_peaks()
-    int8_peak = 2.0 * peaks["bf16_tflops"]
+    8192^3, median of 5 launches per nesting, against the INT8 ceiling; outputs checked equal to the full-bit GEMM's."""
     S = 8192
     gen = torch.Generator(device=dev)
     gen.manual_seed(11)
@@ -473,8 +626,40 @@ def _nested_rows(nq, torch, dev):
                 ts.append(a.elapsed_time(b))
         ms = float(np.median(ts))
         t = 2.0 * S * S * S / (ms * 1e-3) / 1e12
-        out[f"h{h}"] = {"tops": round(t, 1), "frac_int8_peak": round(t / int8_peak, 3), "ms": round(ms, 4),
+        out[f"h{h}"] = {"tops": round(t, 1), "ms": round(ms, 4), **_frac(t, peaks),
                         "weight_bytes_per_element": (N_BITS + 1) / 8, "equals_full_bit": bool(torch.equal(y, ref))}
+    return out
+
+
+def _output_type_rows(nq, torch, state, sizes, peaks):
+    """Config 4 with the other two output types, timed once each (median of 3 launches after a warm-up launch):
+    fp32 Y, and the raw INT32 accumulators with no Y.  Full-bit and part-bit h = 6."""
+    out = {}
+    for s in sizes:
+        d = state[s]
+        y32 = torch.empty((s, s), dtype=torch.float32, device=d["X"].device)
+        acc = torch.empty((s, s), dtype=torch.int32, device=d["X"].device)
+        row = {}
+        for name, fn in (
+                ("full_fp32", lambda: nq.nq_gemm_full(d["X"], d["w_rec"], d["w_scale"], ACT_SCALE, y_out=y32)),
+                ("part_h6_fp32", lambda: nq.nq_gemm_part(d["X"], d["hi"][6], s, N_BITS, 6, d["w_scale"], ACT_SCALE, y_out=y32)),
+                ("full_int32", lambda: nq.nq_gemm_full(d["X"], d["w_rec"], d["w_scale"], ACT_SCALE, acc_out=acc, y_dtype=None)),
+                ("part_h6_int32", lambda: nq.nq_gemm_part(d["X"], d["hi"][6], s, N_BITS, 6, d["w_scale"], ACT_SCALE, acc_out=acc, y_dtype=None))):
+            ts = []
+            for rep in range(4):
+                a = torch.cuda.Event(enable_timing=True)
+                b = torch.cuda.Event(enable_timing=True)
+                a.record()
+                fn()
+                b.record()
+                torch.cuda.synchronize()
+                if rep:
+                    ts.append(a.elapsed_time(b))
+            ms = float(np.median(ts))
+            t = 2.0 * s ** 3 / (ms * 1e-3) / 1e12
+            row[name] = {"tops": round(t, 1), "ms": round(ms, 4), **_frac(t, peaks)}
+        out[str(s)] = row
+        del y32, acc
     return out
 
 
@@ -523,12 +708,81 @@ def _device_conv_weights(torch, L, dev, gen):
     return q[:, :L.K], s.float()
 
 
-def _model_rows(nq, torch, wl, dev, conv_batch):
-    """Configs 3 and 5 through both modes, layer by layer on seeded device-side inputs of the stated shapes and
-    distributions: the ResNet-101-shaped stack (104 convolutions + classifier, batch `conv_batch`, NCHW int8
-    activations ~ U{0..127}, INT8 nesting INT6, bf16 out) and the ViT-B/16 linears (M = 256 * 197 tokens, INT8
-    nesting INT4).  Each layer is timed with its own pair of CUDA events, median of 3 passes; inputs of one pass
-    exceed L2, so nothing is flushed."""
+def time_layers(torch, prepared, call, reps=4):
+    """ms per layer: every layer between its own pair of CUDA events, median over reps - 1 passes (first discarded)."""
+    per_layer = []
+    for rep in range(reps):
+        evs = []
+        for cs in prepared:
+            a = torch.cuda.Event(enable_timing=True)
+            b = torch.cuda.Event(enable_timing=True)
+            a.record()
+            call(cs)
+            b.record()
+            evs.append((a, b))
+        torch.cuda.synchronize()
+        if rep:
+            per_layer.append([a.elapsed_time(b) for a, b in evs])
+    return np.median(np.array(per_layer), axis=0)
+
+
+def capture_stack(torch, prepared, call):
+    """The whole stack as ONE CUDA graph (every launch of every layer, in order), or None when capture fails.  The
+    library calls only enqueue kernels on the current stream, so they can be recorded once and replayed."""
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for cs in prepared:
+                call(cs)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for cs in prepared:
+                call(cs)
+        return g
+    except Exception:
+        torch.cuda.synchronize()
+        return None
+
+
+def time_graph(torch, g, reps=6):
+    ts = []
+    for rep in range(reps):
+        a = torch.cuda.Event(enable_timing=True)
+        b = torch.cuda.Event(enable_timing=True)
+        a.record()
+        g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        if rep:
+            ts.append(a.elapsed_time(b))
+    return float(np.median(ts))
+
+
+def stack_row(torch, prepared, call, ops, roofline_us, graph=True):
+    """One variant of a stack: layer by layer (sum of per-layer medians) and as one graph launch."""
+    ms_layers = time_layers(torch, prepared, call)
+    row = {"ms": round(float(ms_layers.sum()), 3), "tops": round(ops / (float(ms_layers.sum()) * 1e-3) / 1e12, 1),
+           "roofline_sum_ms": round(roofline_us / 1e3, 3), "frac_roofline": round(roofline_us / 1e3 / float(ms_layers.sum()), 3)}
+    if graph:
+        g = capture_stack(torch, prepared, call)
+        if g is not None:
+            gms = time_graph(torch, g)
+            row["graph_ms"] = round(gms, 3)
+            row["graph_frac_roofline"] = round(roofline_us / 1e3 / gms, 3)
+            del g
+    return row, ms_layers
+
+
+def _model_rows(nq, torch, wl, dev, conv_batch, peaks):
+    """Configs 3 and 5 through both modes on seeded device-side inputs of the stated shapes and distributions: the
+    ResNet-101-shaped stack (104 convolutions + classifier, batch `conv_batch`, int8 activations ~ U{0..127}, INT8
+    nesting INT6) and the ViT-B/16 linears (M = 256 * 197 tokens, INT8 nesting INT4).  Every variant is timed layer by
+    layer (own pair of CUDA events per layer, median of 3 passes) and as one CUDA-graph launch of the whole stack;
+    inputs of one pass exceed L2, so nothing is flushed.  `frac_roofline` = sum over layers of max(ops / INT8 ceiling,
+    algorithmic bytes / HBM copy bandwidth) over the measured time."""
     gen = torch.Generator(device=dev)
     gen.manual_seed(wl.BASE_SEED + 3000)
     out = {}
@@ -536,104 +790,82 @@ def _model_rows(nq, torch, wl, dev, conv_batch):
     layers = wl.resnet101_layers()
     xs, prepared = {}, []
     y_elems = max(conv_batch * L.Ho * L.Wo * L.Cout for L in layers)
-    ybuf = torch.empty(y_elems, dtype=torch.bfloat16, device=dev)
+    ybuf = torch.empty(y_elems, dtype=torch.float32, device=dev)
     work_bytes = 0
     for L in layers:
         key = (L.Cin, L.H, L.W)
         if key not in xs:
             xs[key] = torch.randint(0, 128, (conv_batch, L.Cin, L.H, L.W), dtype=torch.int8, device=dev, generator=gen)
-        desc = nq.nq_conv_desc(conv_batch, L.Cin, L.H, L.W, L.Cout, L.R, L.S, L.stride, L.pad, 1)
+            xs[("nhwc",) + key] = xs[key].permute(0, 2, 3, 1).contiguous()
+        args5 = (conv_batch, L.Cin, L.H, L.W, L.Cout, L.R, L.S, L.stride, L.pad)
+        desc = nq.nq_conv_desc(*args5, 1)
+        desc_nhwc = nq.nq_conv_desc(*args5, 0)
         w, ws = _device_conv_weights(torch, L, dev, gen)
         m = torch.randint(0, 2, (L.Cout, w.stride(0)), dtype=torch.uint8, device=dev, generator=gen)[:, :L.K]
         hi, lo = nq.nq_decompose(w, m, N_BITS, CONV_H, True)
-        work_bytes = max(work_bytes, nq.nq_conv_workspace_bytes(desc))
-        prepared.append({"desc": desc, "w": w, "hi": hi, "lo": lo, "ws": ws, "x": xs[key], "act": 0.02,
-                         "y": ybuf[:conv_batch * L.Ho * L.Wo * L.Cout].view(conv_batch, L.Ho, L.Wo, L.Cout)})
+        work_bytes = max(work_bytes, nq.nq_conv_workspace_bytes(desc), nq.nq_conv_workspace_bytes(desc_nhwc))
+        n_out = conv_batch * L.Ho * L.Wo * L.Cout
+        shape = (conv_batch, L.Ho, L.Wo, L.Cout)
+        prepared.append({"L": L, "desc": desc, "desc_nhwc": desc_nhwc, "w": w, "hi": hi, "lo": lo, "ws": ws, "x": xs[key],
+                         "x_nhwc": xs[("nhwc",) + key], "act": 0.02,
+                         "y": ybuf.view(torch.bfloat16)[:n_out].view(shape), "y32": ybuf[:n_out].view(shape),
+                         "yq": ybuf.view(torch.int8)[:n_out].view(shape)})
     work = torch.empty(work_bytes + 2048, dtype=torch.uint8, device=dev)
     for cs in prepared:
         cs["work"] = work
     ops = sum(2.0 * float(np.prod(L.gemm_view(conv_batch))) for L in layers)
+
+    def roof(part, esize):
+        return sum(conv_roofline_us(L, conv_batch, part, CONV_H, esize, peaks) for L in layers)
+
+    def conv(cs, part, nhwc, y):
+        nq.nq_conv_implicit_gemm(cs["x_nhwc"] if nhwc else cs["x"], cs["hi"] if part else cs["w"],
+                                 cs["desc_nhwc"] if nhwc else cs["desc"], cs["ws"], cs["act"], part_bit=part, n_bits=N_BITS,
+                                 h_bits=CONV_H, workspace=cs["work"], y_out=cs[y])
+
     res = {}
+    per_layer_nhwc = None
     for part in (False, True):
-        per_layer = []
-        for rep in range(4):
-            evs = []
-            for cs in prepared:
-                a = torch.cuda.Event(enable_timing=True)
-                b = torch.cuda.Event(enable_timing=True)
-                a.record()
-                _run_conv(nq, cs, part)
-                b.record()
-                evs.append((a, b))
-            torch.cuda.synchronize()
-            if rep:
-                per_layer.append([a.elapsed_time(b) for a, b in evs])
-        ms = float(np.sum(np.median(np.array(per_layer), axis=0)))
-        res["part_bit" if part else "full_bit"] = {"ms": round(ms, 3), "tops": round(ops / (ms * 1e-3) / 1e12, 1)}
+        mode = "part_bit" if part else "full_bit"
+        res[mode], _ = stack_row(torch, prepared, lambda cs: conv(cs, part, False, "y"), ops, roof(part, 2))
+        res[mode + "_nhwc_in"], ms_l = stack_row(torch, prepared, lambda cs: conv(cs, part, True, "y"), ops, roof(part, 2))
+        if not part:
+            per_layer_nhwc = ms_l
+        # what the NCHW -> NHWC pre-pass (a transposing kernel in front of every layer) costs: the difference
+        res[mode]["nchw_prepass_ms"] = round(res[mode]["ms"] - res[mode + "_nhwc_in"]["ms"], 3)
+    res["full_bit_nhwc_in_fp32_out"], _ = stack_row(torch, prepared, lambda cs: conv(cs, False, True, "y32"), ops, roof(False, 4))
     # the full-bit stack again with no INT8 copy of the weights: every layer rebuilds them from the two packed parts
-    per_layer = []
-    for rep in range(4):
-        evs = []
-        for cs in prepared:
-            a = torch.cuda.Event(enable_timing=True)
-            b = torch.cuda.Event(enable_timing=True)
-            a.record()
-            nq.nq_conv_implicit_gemm_nested(cs["x"], cs["hi"], cs["lo"], cs["desc"], cs["ws"], cs["act"], n_bits=N_BITS,
-                                            h_bits=CONV_H, workspace=cs["work"], y_out=cs["y"])
-            b.record()
-            evs.append((a, b))
-        torch.cuda.synchronize()
-        if rep:
-            per_layer.append([a.elapsed_time(b) for a, b in evs])
-    ms = float(np.sum(np.median(np.array(per_layer), axis=0)))
-    res["nested_full_bit"] = {"ms": round(ms, 3), "tops": round(ops / (ms * 1e-3) / 1e12, 1)}
+    res["nested_full_bit"], _ = stack_row(
+        torch, prepared, lambda cs: nq.nq_conv_implicit_gemm_nested(cs["x"], cs["hi"], cs["lo"], cs["desc"], cs["ws"], cs["act"],
+                                                                    n_bits=N_BITS, h_bits=CONV_H, workspace=cs["work"], y_out=cs["y"]),
+        ops, roof(False, 2), graph=False)
+    # chained form: NHWC int8 activations in, the next layer's INT8 activations out (requantising epilogue with ReLU),
+    # no layout pre-pass; every layer still runs on its own input
+    for part in (False, True):
+        res["chained_int8_out_" + ("part_bit" if part else "full_bit")], _ = stack_row(
+            torch, prepared, lambda cs: nq.nq_conv_implicit_gemm_q8(cs["x_nhwc"], cs["hi"] if part else cs["w"], cs["desc_nhwc"],
+                                                                    cs["ws"], cs["act"], 0.5, relu=True, part_bit=part, n_bits=N_BITS,
+                                                                    h_bits=CONV_H, workspace=cs["work"], y_out=cs["yq"]),
+            ops, roof(part, 1))
+    res["chained_int8_out_nested_full_bit"], _ = stack_row(
+        torch, prepared, lambda cs: nq.nq_conv_implicit_gemm_nested_q8(cs["x_nhwc"], cs["hi"], cs["lo"], cs["desc_nhwc"], cs["ws"],
+                                                                       cs["act"], 0.5, relu=True, n_bits=N_BITS, h_bits=CONV_H,
+                                                                       workspace=cs["work"], y_out=cs["yq"]),
+        ops, roof(False, 1), graph=False)
+    # per distinct layer shape, full-bit, NHWC in, bf16 out: where the stack's time goes against each layer's roofline
+    shapes = {}
+    for cs, ms in zip(prepared, per_layer_nhwc):
+        L = cs["L"]
+        key = (L.Cin, L.H, L.Cout, L.R, L.stride)
+        e = shapes.setdefault(key, {"first": L.name, "count": 0, "ms": 0.0,
+                                    "roofline_us": round(conv_roofline_us(L, conv_batch, False, CONV_H, 2, peaks), 2)})
+        e["count"] += 1
+        e["ms"] += float(ms)
+    res["per_shape_full_bit_nhwc_in"] = [
+        {"first": e["first"], "count": e["count"], "us_each": round(1e3 * e["ms"] / e["count"], 1), "roofline_us": e["roofline_us"],
+         "frac_roofline": round(e["roofline_us"] / (1e3 * e["ms"] / e["count"]), 3)} for e in shapes.values()]
     res.update({"layers": len(layers), "batch": conv_batch, "weights": sum(L.weights for L in layers),
                 "tera_ops_per_pass": round(ops / 1e12, 3)})
-    # the same stack in chained form: NHWC int8 activations in, the next layer's INT8 activations out (requantising
-    # epilogue with ReLU), no layout pre-pass; every layer still runs on its own input
-    yq = torch.empty(y_elems, dtype=torch.int8, device=dev)
-    for cs, L in zip(prepared, layers):
-        key = ("nhwc", L.Cin, L.H, L.W)
-        if key not in xs:
-            xs[key] = cs["x"].permute(0, 2, 3, 1).contiguous()
-        cs["x_nhwc"] = xs[key]
-        cs["desc_nhwc"] = nq.nq_conv_desc(conv_batch, L.Cin, L.H, L.W, L.Cout, L.R, L.S, L.stride, L.pad, 0)
-        cs["yq"] = yq[:conv_batch * L.Ho * L.Wo * L.Cout].view(conv_batch, L.Ho, L.Wo, L.Cout)
-    for part in (False, True):
-        per_layer = []
-        for rep in range(4):
-            evs = []
-            for cs in prepared:
-                a = torch.cuda.Event(enable_timing=True)
-                b = torch.cuda.Event(enable_timing=True)
-                a.record()
-                nq.nq_conv_implicit_gemm_q8(cs["x_nhwc"], cs["hi"] if part else cs["w"], cs["desc_nhwc"], cs["ws"], cs["act"],
-                                            0.5, relu=True, part_bit=part, n_bits=N_BITS, h_bits=CONV_H,
-                                            workspace=cs["work"], y_out=cs["yq"])
-                b.record()
-                evs.append((a, b))
-            torch.cuda.synchronize()
-            if rep:
-                per_layer.append([a.elapsed_time(b) for a, b in evs])
-        ms = float(np.sum(np.median(np.array(per_layer), axis=0)))
-        res["chained_int8_out_" + ("part_bit" if part else "full_bit")] = {"ms": round(ms, 3), "tops": round(ops / (ms * 1e-3) / 1e12, 1)}
-    per_layer = []
-    for rep in range(4):
-        evs = []
-        for cs in prepared:
-            a = torch.cuda.Event(enable_timing=True)
-            b = torch.cuda.Event(enable_timing=True)
-            a.record()
-            nq.nq_conv_implicit_gemm_nested_q8(cs["x_nhwc"], cs["hi"], cs["lo"], cs["desc_nhwc"], cs["ws"], cs["act"], 0.5,
-                                               relu=True, n_bits=N_BITS, h_bits=CONV_H, workspace=cs["work"], y_out=cs["yq"])
-            b.record()
-            evs.append((a, b))
-        torch.cuda.synchronize()
-        if rep:
-            per_layer.append([a.elapsed_time(b) for a, b in evs])
-    ms = float(np.sum(np.median(np.array(per_layer), axis=0)))
-    res["chained_int8_out_nested_full_bit"] = {"ms": round(ms, 3), "tops": round(ops / (ms * 1e-3) / 1e12, 1)}
-    del yq
     out["resnet101_stack_int8_6"] = res
     nq.nq_device_status()
     del prepared, xs, ybuf, work
@@ -653,8 +885,8 @@ def _model_rows(nq, torch, wl, dev, conv_batch):
         hi, _ = nq.nq_decompose(w, m, N_BITS, 4, True)
         y = torch.empty((M, n), dtype=torch.bfloat16, device=dev)
         row = {}
-        for name, fn in (("full_bit", lambda: nq.nq_gemm_full(x, w, sc, ACT_SCALE, y_out=y)),
-                         ("part_bit", lambda: nq.nq_gemm_part(x, hi, n, N_BITS, 4, sc, ACT_SCALE, y_out=y))):
+        for name, part, fn in (("full_bit", False, lambda: nq.nq_gemm_full(x, w, sc, ACT_SCALE, y_out=y)),
+                               ("part_bit", True, lambda: nq.nq_gemm_part(x, hi, n, N_BITS, 4, sc, ACT_SCALE, y_out=y))):
             ts = []
             for rep in range(5):
                 a = torch.cuda.Event(enable_timing=True)
@@ -666,7 +898,9 @@ def _model_rows(nq, torch, wl, dev, conv_batch):
                 if rep:
                     ts.append(a.elapsed_time(b))
             ms = float(np.median(ts))
-            row[name] = {"ms": round(ms, 4), "tops": round(2.0 * M * n * k / (ms * 1e-3) / 1e12, 1)}
+            roof_us = layer_roofline_us(M, n, k, M * k, n * k * (0.5 if part else 1.0), M * n * 2, peaks)
+            row[name] = {"ms": round(ms, 4), "tops": round(2.0 * M * n * k / (ms * 1e-3) / 1e12, 1),
+                         "roofline_us": round(roof_us, 1), "frac_roofline": round(roof_us / (ms * 1e3), 3)}
         res[f"K{k}_N{n}"] = row
     res["M"] = M
     out["vit_b16_linears_int8_4"] = res
@@ -802,7 +1036,11 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--conv-batch", type=int, default=32)
     ap.add_argument("--no-conv", dest="conv", action="store_false")
+    ap.add_argument("--no-graphs", dest="graphs", action="store_false",
+                    help="run the convolution stacks of the timed steps layer by layer instead of as CUDA graphs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-ceiling", dest="ceiling", action="store_false",
+                    help="skip the 2 s measurement of the INT8 tensor ceiling (fractions then use 2 x bf16 sustained)")
     ap.add_argument("--no-model-switch", dest="model_switch", action="store_false")
     ap.add_argument("--no-model-rows", dest="model_rows", action="store_false",
                     help="skip the ResNet-101-shaped stack and the ViT-B linears (timed after the steps)")
@@ -826,7 +1064,9 @@ def main():
             import torch
             import paper_2506_17870_b200 as nq
             torch.cuda.set_device(local_rank)
-            print(json.dumps({"rows": {"gemm_nested_8192": _nested_rows(nq, torch, torch.device("cuda", local_rank))}}), flush=True)
+            pk = measured_peaks()
+            pk["int8_tops"], pk["int8_source"] = 2.0 * pk["bf16_tflops_sustained"], "2 x bf16 sustained"
+            print(json.dumps({"rows": {"gemm_nested_8192": _nested_rows(nq, torch, torch.device("cuda", local_rank), pk)}}), flush=True)
         return
 
     if world > 1:

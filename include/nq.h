@@ -300,6 +300,19 @@ NQ_API int nq_conv_implicit_gemm_static(const int8_t *X, const void *Wt, int64_t
                                         const float *bias, int32_t *acc_out, void *Y, int y_dtype, void *stream);
 
 /*
+ * Measurement aid (the paper has no counterpart: it times no integer kernel).  Enqueues ONE launch of a kernel
+ * that only issues the tensor instruction of the GEMM / convolution kernels -- tcgen05.mma kind::i8 on CTA pairs,
+ * 256 x 256 x 32 per instruction -- on operands that already sit in shared memory (small signed pseudo-random
+ * bytes), accumulating in tensor memory: no global loads, no epilogue.  Every CTA pair (one per two SMs) runs
+ * stage_iters stages of four instructions.  Timed with CUDA events by the caller, ops / time is the ceiling of
+ * the INT8 tensor path on this GPU under its power limit, the denominator of the GEMM roofline.
+ *   stage_iters  in [1, 2^21] (a launch of 3700 stages lasts about a millisecond)
+ *   ops_out (host, out, may be NULL)  integer operations of the launch: pairs * stage_iters * 4 * 2*256*256*32
+ * Allocates nothing; the wait at its end is bounded like every other (nq_device_status).
+ */
+NQ_API int nq_i8_mma_ceiling(int64_t stage_iters, double *ops_out, void *stream);
+
+/*
  * Every on-device wait in the GEMM / convolution kernels is bounded.  If one expires the kernel
  * records it and returns instead of hanging.  This call synchronises `stream`, reads and clears
  * the record of the current device: returns NQ_OK, NQ_ERR_TIMEOUT (with *where_out = an internal

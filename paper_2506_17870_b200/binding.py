@@ -31,6 +31,7 @@ EXPORTS = (
     "nq_conv_implicit_gemm_static",
     "nq_gemm_full_q8", "nq_gemm_part_q8", "nq_conv_implicit_gemm_q8", "nq_gemm_nested", "nq_conv_implicit_gemm_nested", "nq_gemm_nested_q8",
     "nq_conv_implicit_gemm_nested_q8",
+    "nq_i8_mma_ceiling",
     "nq_device_status",
 )
 
@@ -509,6 +510,13 @@ def nq_conv_implicit_gemm_static(X: torch.Tensor, Wt: torch.Tensor, desc: nq_con
                                               _y_dtype(y_out.dtype) if y_out is not None else NQ_F32, _stream()),
            "nq_conv_implicit_gemm_static")
     return acc_out, y_out
+
+
+def nq_i8_mma_ceiling(stage_iters: int) -> float:
+    """Enqueues one launch of the MMA-issue-only kernel on the current stream; returns its integer operations."""
+    ops = ctypes.c_double(0.0)
+    _check(lib().nq_i8_mma_ceiling(_i64(stage_iters), ctypes.byref(ops), _stream()), "nq_i8_mma_ceiling")
+    return float(ops.value)
 
 
 def nq_device_status() -> int:
