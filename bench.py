@@ -430,6 +430,10 @@ def run_ours(args, rank, world, local_rank):
         line["rows"]["gemm_output_types_config4"] = _output_type_rows(nq, torch, state, sizes, peaks)
     if model_rows is not None:
         line["rows"].update(model_rows)
+    if have_conv and args.chains:
+        line["rows"]["resnet18_chain_int8_6"] = _chain_rows(nq, torch, wl, dev, peaks, wl.resnet18_layers(), 2, args.conv_batch)
+        if args.model_rows:
+            line["rows"]["resnet101_chain_int8_6"] = _chain_rows(nq, torch, wl, dev, peaks, wl.resnet101_layers(), 3, args.model_batch)
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(sizes, host, args.cpu_rows)
     return line
@@ -543,6 +547,60 @@ def _config2_rows(nq, torch, wl, conv_layers, conv_state, conv_batch, peaks, eve
     out["conv_full_stack_nhwc_in_fp32_out"], _ = stack_row(
         torch, nhwc, lambda cs: nq.nq_conv_implicit_gemm(cs["x"], cs["w"], cs["desc"], cs["ws"], cs["act"], part_bit=False,
                                                          workspace=cs["work"], y_out=cs["y32"]), ops, roof)
+    return out
+
+
+def _chain_rows(nq, torch, wl, dev, peaks, layers, config, batch):
+    """A ResNet-shaped model as ONE dependent chain on the device (stem, max pooling, residual blocks with the skip
+    tensor added in the epilogue, global average pooling, classifier): INT8 activations hand over between layers, NCHW
+    int8 input.  Scales are calibrated on the device first (set-up).  Timed per pass, layer by layer launches and as
+    one CUDA-graph launch, in full-bit, part-bit and nested full-bit mode; the roofline of a pass is the sum over layers
+    of max(ops / INT8 ceiling, (input + weights + INT8 output + skip tensor) / HBM) plus the pooling passes' bytes."""
+    from paper_2506_17870_b200.chain import ResNetChain
+    plan = wl.resnet_chain_plan(layers)
+    weights = wl.chain_weights(config, layers)
+    model = ResNetChain(layers, plan, weights, batch, 0.02, n_bits=N_BITS, h_bits=CONV_H, device=dev)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(wl.BASE_SEED + 7000 + config)
+    x = torch.randint(0, 128, (batch, 3, 224, 224), dtype=torch.int8, device=dev, generator=gen)
+    by = {L.name: L for L in layers}
+    ops = 0.0
+    out = {"batch": batch, "steps": len(plan), "kernels_per_pass": model.kernels_per_pass()}
+    for mode in ("full", "part", "nested"):
+        model.calibrate(x, "part" if mode == "part" else "full")
+        wbytes = {"full": 1.0, "part": CONV_H / 8.0, "nested": (N_BITS + 1) / 8.0}[mode]
+        roof, ops = 0.0, 0.0
+        for st in plan:
+            if st["op"] in ("conv", "fc"):
+                L = by[st["layer"]]
+                M, N, K = L.gemm_view(batch)
+                ops += 2.0 * M * N * K
+                out_b = M * N * (4 if st["op"] == "fc" else 1) + (M * N if st.get("skip") else 0)
+                roof += layer_roofline_us(M, N, K, batch * L.Cin * L.H * L.W, N * K * wbytes, out_b, peaks)
+            else:
+                roof += 1e6 * (model.t[st["src"]].numel() + model.t[st["dst"]].numel()) / (peaks["hbm_gbs"] * 1e9)
+        ts = []
+        for rep in range(5):
+            a = torch.cuda.Event(enable_timing=True)
+            b = torch.cuda.Event(enable_timing=True)
+            a.record()
+            model.run(x, mode)
+            b.record()
+            torch.cuda.synchronize()
+            if rep:
+                ts.append(a.elapsed_time(b))
+        ms = float(np.median(ts))
+        row = {"ms": round(ms, 3), "tops": round(ops / (ms * 1e-3) / 1e12, 1), "roofline_sum_ms": round(roof / 1e3, 3),
+               "frac_roofline": round(roof / 1e3 / ms, 3)}
+        g = capture_stack(torch, [None], lambda _: model.run(x, mode))
+        if g is not None:
+            gms = time_graph(torch, g)
+            row["graph_ms"] = round(gms, 3)
+            row["graph_frac_roofline"] = round(roof / 1e3 / gms, 3)
+            del g
+        out[mode] = row
+    nq.nq_device_status()
+    out["tera_ops_per_pass"] = round(ops / 1e12, 3)
     return out
 
 
@@ -1045,6 +1103,8 @@ def main():
     ap.add_argument("--no-model-rows", dest="model_rows", action="store_false",
                     help="skip the ResNet-101-shaped stack and the ViT-B linears (timed after the steps)")
     ap.add_argument("--model-batch", type=int, default=128)
+    ap.add_argument("--no-chains", dest="chains", action="store_false",
+                    help="skip the dependent-chain rows (ResNet-18-shaped at --conv-batch, ResNet-101-shaped at --model-batch)")
     ap.add_argument("--nested-only", action="store_true",
                     help="time only the nested full-bit GEMM rows (8192^3, h in {4..7}) and print them")
     args = ap.parse_args()

@@ -274,6 +274,46 @@ NQ_API int nq_conv_implicit_gemm_nested_q8(const int8_t *X, const void *packed_h
 
 
 /*
+ * Pieces a chained model needs between its layers.  The paper runs its models with 8-bit activations but defines
+ * none of this arithmetic (how a block's skip path, or a pooling layer, treats the INT8 tensors), so these are the
+ * library's own definitions, all in fp32 with one rounding per operation:
+ *
+ * Residual blocks -- the requantising convolution (nq_conv_implicit_gemm_q8, and its nested full-bit form) with a
+ * skip tensor added before the activation:
+ *   v = dequantised convolution output (+ bias[j]);   v = fl(v + fl(float(residual[m, j]) * residual_scale))
+ *   v = max(v, 0) when relu != 0;   q = clip(round_half_even(fl(v * fl(1 / out_scale))), -128, 127)
+ *   residual (device) int8, the output's shape [B, Ho, Wo, Cout], dense NHWC: the block's input (identity skip) or
+ *   the requantised output of its 1 x 1 down-sampling convolution; residual_scale is that tensor's activation scale.
+ *   A 16-byte aligned residual with Cout a multiple of 16 takes the fast path; anything else is read byte-wise.
+ *   Every other argument is that of nq_conv_implicit_gemm_q8 / nq_conv_implicit_gemm_nested_q8.
+ */
+NQ_API int nq_conv_implicit_gemm_q8_res(const int8_t *X, const void *Wt, int64_t ldw, int part_bit, int n_bits, int h_bits,
+                                 const nq_conv_desc *desc, const float *w_scale, float act_scale, const float *bias,
+                                 const int8_t *residual, float residual_scale, float out_scale, int relu, int8_t *Yq,
+                                 void *workspace, int64_t workspace_bytes, void *stream);
+NQ_API int nq_conv_implicit_gemm_nested_q8_res(const int8_t *X, const void *packed_high, const void *packed_low,
+                                        int n_bits, int h_bits, const nq_conv_desc *desc, const float *w_scale,
+                                        float act_scale, const float *bias, const int8_t *residual,
+                                        float residual_scale, float out_scale, int relu, int8_t *Yq,
+                                        void *workspace, int64_t workspace_bytes, void *stream);
+
+/*
+ * Max pooling of INT8 NHWC activations [B, H, W, C] -> [B, Ho, Wo, C], Ho = (H + 2*pad - ksize) / stride + 1:
+ * the integer maximum over the window's taps that lie inside the image (padding never wins); the activation scale
+ * is unchanged.  pad < ksize.  C a multiple of 16 with 16-byte aligned tensors takes 16-byte accesses.
+ */
+NQ_API int nq_maxpool_nhwc_i8(const int8_t *X, int B, int H, int W, int C, int ksize, int stride, int pad, int8_t *Y,
+                       void *stream);
+
+/*
+ * Global average pooling with requantisation, INT8 NHWC [B, H, W, C] -> INT8 [B, C]:
+ *   sum = integer sum over the H*W pixels;  a = fl(in_scale / float(H*W));
+ *   q = clip(round_half_even(fl(fl(float(sum) * a) * fl(1 / out_scale))), -128, 127)
+ */
+NQ_API int nq_avgpool_requant_nhwc_i8(const int8_t *X, int B, int H, int W, int C, float in_scale, float out_scale,
+                               int8_t *Y, void *stream);
+
+/*
  * The convolution again, for callers that must not allocate.  (The paper has no counterpart; this is a
  * convenience of the library.)  nq_conv_implicit_gemm needs a workspace whenever it re-lays the input
  * (NCHW activations, or a channel count it cannot gather in place), and somebody has to allocate that.
@@ -298,6 +338,16 @@ NQ_API int nq_conv_implicit_gemm_nested_q8(const int8_t *X, const void *packed_h
 NQ_API int nq_conv_implicit_gemm_static(const int8_t *X, const void *Wt, int64_t ldw, int part_bit, int n_bits,
                                         int h_bits, const nq_conv_desc *desc, const float *w_scale, float act_scale,
                                         const float *bias, int32_t *acc_out, void *Y, int y_dtype, void *stream);
+
+/*
+ * Test aid (the paper has no counterpart).  The GEMM / convolution kernels have two pairs of equivalent code paths:
+ * outputs written by TMA tile stores or by ordinary stores, and part-bit fields of 1, 2 and 4 bits read straight
+ * from the packed matrix or through the shared-memory ring of packed tiles.  The library picks by alignment and
+ * field width; this switch forces the second of each pair so that a test can compare the two bit for bit.
+ * Process-wide and not synchronised: set it only while no call of another thread is in flight.
+ */
+enum { NQ_DEBUG_PLAIN_STORES = 0, NQ_DEBUG_PACKED_RING = 1 };
+NQ_API int nq_debug_set(int which, int enabled);
 
 /*
  * Measurement aid (the paper has no counterpart: it times no integer kernel).  Enqueues ONE launch of a kernel

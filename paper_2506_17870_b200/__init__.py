@@ -12,5 +12,7 @@ from .binding import (  # noqa: F401
     nq_word64_row_words, nq_word64_to_sliced, nq_sliced_to_word64,
     nq_gemm_full_q8, nq_gemm_part_q8, nq_conv_implicit_gemm_q8, nq_gemm_nested, nq_conv_implicit_gemm_nested, nq_gemm_nested_q8,
     nq_conv_implicit_gemm_nested_q8,
-    nq_i8_mma_ceiling, nq_rounding_mask, NQ_ROUND_DOWN, NQ_ROUND_UP, NQ_ROUND_NEAREST,
+    nq_i8_mma_ceiling, nq_debug_set, NQ_DEBUG_PLAIN_STORES, NQ_DEBUG_PACKED_RING,
+    nq_conv_implicit_gemm_q8_res, nq_conv_implicit_gemm_nested_q8_res, nq_maxpool_nhwc_i8, nq_avgpool_requant_nhwc_i8,
+    nq_rounding_mask, NQ_ROUND_DOWN, NQ_ROUND_UP, NQ_ROUND_NEAREST,
 )

@@ -9,14 +9,13 @@ raises ``NqLibraryError``.
 from __future__ import annotations
 
 import ctypes
-import os
 from pathlib import Path
 from typing import Optional, Sequence
 
 import torch
 
 _PKG = Path(__file__).resolve().parent
-_LIB_PATH = Path(os.environ.get("NQ_B200_LIB", _PKG / "libnq_b200.so"))   # override: a differently built copy
+_LIB_PATH = _PKG / "libnq_b200.so"
 _lib = None
 
 NQ_OK = 0
@@ -31,7 +30,8 @@ EXPORTS = (
     "nq_conv_implicit_gemm_static",
     "nq_gemm_full_q8", "nq_gemm_part_q8", "nq_conv_implicit_gemm_q8", "nq_gemm_nested", "nq_conv_implicit_gemm_nested", "nq_gemm_nested_q8",
     "nq_conv_implicit_gemm_nested_q8",
-    "nq_i8_mma_ceiling",
+    "nq_i8_mma_ceiling", "nq_debug_set",
+    "nq_conv_implicit_gemm_q8_res", "nq_conv_implicit_gemm_nested_q8_res", "nq_maxpool_nhwc_i8", "nq_avgpool_requant_nhwc_i8",
     "nq_device_status",
 )
 
@@ -417,6 +417,58 @@ def nq_conv_implicit_gemm_nested_q8(X: torch.Tensor, packed_high: torch.Tensor, 
     return y
 
 
+def nq_conv_implicit_gemm_q8_res(X: torch.Tensor, Wt: torch.Tensor, desc: nq_conv_desc, w_scale: torch.Tensor, act_scale: float,
+                                 residual: torch.Tensor, residual_scale: float, out_scale: float, relu: bool = True,
+                                 part_bit: bool = False, n_bits: int = 8, h_bits: int = 6,
+                                 bias: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                                 y_out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Requantising convolution with a residual connection: `residual` (int8, the output's NHWC shape, scale
+    residual_scale) is added, dequantised, before the activation."""
+    Ho = (desc.H + 2 * desc.pad - desc.R) // desc.stride + 1
+    Wo = (desc.W + 2 * desc.pad - desc.S) // desc.stride + 1
+    _need(residual, torch.int8, "residual")
+    if tuple(residual.shape) != (desc.B, Ho, Wo, desc.Cout) or not residual.is_contiguous():
+        raise ValueError("residual must be a dense NHWC tensor of the output's shape")
+    need = nq_conv_workspace_bytes(desc)
+    if workspace is None:
+        workspace = torch.empty(max(need, 0) + 2048, dtype=torch.uint8, device=X.device)
+    off = (-workspace.data_ptr()) % 1024
+    y = y_out if y_out is not None else torch.empty((desc.B, Ho, Wo, desc.Cout), dtype=torch.int8, device=X.device)
+    ldw = _ld(Wt) if not part_bit else 0
+    _check(lib().nq_conv_implicit_gemm_q8_res(_ptr(X), _ptr(Wt), _i64(ldw), int(bool(part_bit)), n_bits, h_bits,
+                                              ctypes.byref(desc), _ptr(w_scale), ctypes.c_float(act_scale), _ptr(bias),
+                                              _ptr(residual), ctypes.c_float(residual_scale), ctypes.c_float(out_scale),
+                                              int(bool(relu)), _ptr(y), ctypes.c_void_p(workspace.data_ptr() + off),
+                                              _i64(workspace.numel() - off), _stream()), "nq_conv_implicit_gemm_q8_res")
+    return y
+
+
+def nq_conv_implicit_gemm_nested_q8_res(X: torch.Tensor, packed_high: torch.Tensor, packed_low: torch.Tensor,
+                                        desc: nq_conv_desc, w_scale: torch.Tensor, act_scale: float,
+                                        residual: torch.Tensor, residual_scale: float, out_scale: float,
+                                        relu: bool = True, n_bits: int = 8, h_bits: int = 6,
+                                        bias: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                                        y_out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """The same in nested full-bit mode (weights rebuilt from the two packed parts inside the kernel)."""
+    Ho = (desc.H + 2 * desc.pad - desc.R) // desc.stride + 1
+    Wo = (desc.W + 2 * desc.pad - desc.S) // desc.stride + 1
+    _need(residual, torch.int8, "residual")
+    if tuple(residual.shape) != (desc.B, Ho, Wo, desc.Cout) or not residual.is_contiguous():
+        raise ValueError("residual must be a dense NHWC tensor of the output's shape")
+    need = nq_conv_workspace_bytes(desc)
+    if workspace is None:
+        workspace = torch.empty(max(need, 0) + 2048, dtype=torch.uint8, device=X.device)
+    off = (-workspace.data_ptr()) % 1024
+    y = y_out if y_out is not None else torch.empty((desc.B, Ho, Wo, desc.Cout), dtype=torch.int8, device=X.device)
+    _check(lib().nq_conv_implicit_gemm_nested_q8_res(_ptr(X), _ptr(packed_high), _ptr(packed_low), n_bits, h_bits,
+                                                     ctypes.byref(desc), _ptr(w_scale), ctypes.c_float(act_scale), _ptr(bias),
+                                                     _ptr(residual), ctypes.c_float(residual_scale), ctypes.c_float(out_scale),
+                                                     int(bool(relu)), _ptr(y), ctypes.c_void_p(workspace.data_ptr() + off),
+                                                     _i64(workspace.numel() - off), _stream()),
+           "nq_conv_implicit_gemm_nested_q8_res")
+    return y
+
+
 def nq_conv_workspace_bytes(desc: nq_conv_desc) -> int:
     return int(lib().nq_conv_workspace_bytes(ctypes.byref(desc)))
 
@@ -510,6 +562,35 @@ def nq_conv_implicit_gemm_static(X: torch.Tensor, Wt: torch.Tensor, desc: nq_con
                                               _y_dtype(y_out.dtype) if y_out is not None else NQ_F32, _stream()),
            "nq_conv_implicit_gemm_static")
     return acc_out, y_out
+
+
+NQ_DEBUG_PLAIN_STORES, NQ_DEBUG_PACKED_RING = 0, 1
+
+
+def nq_debug_set(which: int, enabled: bool) -> None:
+    """Test aid: force ordinary stores / the packed-tile ring (see nq.h)."""
+    _check(lib().nq_debug_set(int(which), int(bool(enabled))), "nq_debug_set")
+
+
+def nq_maxpool_nhwc_i8(X: torch.Tensor, ksize: int, stride: int, pad: int, y_out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """INT8 NHWC [B, H, W, C] -> [B, Ho, Wo, C], integer maximum over the taps inside the image."""
+    _need(X, torch.int8, "X", 4)
+    B, H, W, C = X.shape
+    Ho, Wo = (H + 2 * pad - ksize) // stride + 1, (W + 2 * pad - ksize) // stride + 1
+    y = y_out if y_out is not None else torch.empty((B, Ho, Wo, C), dtype=torch.int8, device=X.device)
+    _check(lib().nq_maxpool_nhwc_i8(_ptr(X), B, H, W, C, ksize, stride, pad, _ptr(y), _stream()), "nq_maxpool_nhwc_i8")
+    return y
+
+
+def nq_avgpool_requant_nhwc_i8(X: torch.Tensor, in_scale: float, out_scale: float,
+                               y_out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """INT8 NHWC [B, H, W, C] -> INT8 [B, C]: global average, requantised."""
+    _need(X, torch.int8, "X", 4)
+    B, H, W, C = X.shape
+    y = y_out if y_out is not None else torch.empty((B, C), dtype=torch.int8, device=X.device)
+    _check(lib().nq_avgpool_requant_nhwc_i8(_ptr(X), B, H, W, C, ctypes.c_float(in_scale), ctypes.c_float(out_scale),
+                                            _ptr(y), _stream()), "nq_avgpool_requant_nhwc_i8")
+    return y
 
 
 def nq_i8_mma_ceiling(stage_iters: int) -> float:

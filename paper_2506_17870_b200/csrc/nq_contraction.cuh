@@ -94,6 +94,9 @@ struct ContractionArgs {
     int y_is_i8;         // requantised INT8 output: q = clip(rint(fl(relu(v) * inv_out_scale)))
     int relu;
     float inv_out_scale;
+    const int8_t* residual;   // requantised output only: INT8 skip tensor [M, N], row pitch ld_res, added dequantised
+    long long ld_res;         //   (fl(float(r) * res_scale)) before the activation; nullptr = none
+    float res_scale;
     unsigned int* status;
 };
 
@@ -333,6 +336,42 @@ __device__ __forceinline__ uint32_t requant4(float v0, float v1, float v2, float
     return out;
 }
 
+// 32 accumulator values of one output row -> dequantised fp32 in the stated rounding order:
+// v = fl(float(acc) * scale_j), then + bias_j with one more rounding.  The 32 factors are the same for every lane:
+// they are read four at a time (a scalar read per column costs a shared-memory wavefront each, and the load/store
+// data path is the busiest unit of this epilogue).
+__device__ __forceinline__ void dequant_chunk(const ContractionArgs& p, const uint32_t (&r)[32], const float* sc,
+                                              const float* bs, float (&v)[32]) {
+#pragma unroll
+    for (int j = 0; j < 32; j += 4) {
+        const float4 s4 = *reinterpret_cast<const float4*>(sc + j);
+        v[j] = __fmul_rn(__int2float_rn((int)r[j]), s4.x);
+        v[j + 1] = __fmul_rn(__int2float_rn((int)r[j + 1]), s4.y);
+        v[j + 2] = __fmul_rn(__int2float_rn((int)r[j + 2]), s4.z);
+        v[j + 3] = __fmul_rn(__int2float_rn((int)r[j + 3]), s4.w);
+    }
+    if (p.bias) {
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) {
+            const float4 b4 = *reinterpret_cast<const float4*>(bs + j);
+            v[j] = __fadd_rn(v[j], b4.x);
+            v[j + 1] = __fadd_rn(v[j + 1], b4.y);
+            v[j + 2] = __fadd_rn(v[j + 2], b4.z);
+            v[j + 3] = __fadd_rn(v[j + 3], b4.w);
+        }
+    }
+}
+
+// The skip path of a residual block: v += fl(float(r) * res_scale), r the INT8 skip values of the same 32 columns
+// (eight words, byte i of word q = column 4q + i).
+__device__ __forceinline__ void add_residual(float (&v)[32], const uint32_t (&w)[8], float res_scale) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        const int r = (int)(int8_t)((w[j >> 2] >> (8 * (j & 3))) & 0xffu);
+        v[j] = __fadd_rn(v[j], __fmul_rn(__int2float_rn(r), res_scale));
+    }
+}
+
 // Epilogue of one thread for 32 consecutive columns of its output row: optional int32 copy (with the
 // part-bit shift), dequantisation in the stated rounding order, fp32 or bf16 store; vector stores when
 // the chunk is whole and the pointers and pitches allow.
@@ -354,26 +393,20 @@ __device__ __forceinline__ void store_chunk(const ContractionArgs& p, long long 
         }
     }
     if (p.y) {
-        // the 32 factors are the same for every lane: read them four at a time (a scalar read per column costs
-        // a shared-memory wavefront each, and the load/store data path is the busiest unit of this epilogue)
         float v[32];
+        dequant_chunk(p, r, sc, bs, v);
+        if (p.residual) {
+            const int8_t* rp = p.residual + row * p.ld_res + col0;
+            uint32_t w[8];
 #pragma unroll
-        for (int j = 0; j < 32; j += 4) {
-            const float4 s4 = *reinterpret_cast<const float4*>(sc + j);
-            v[j] = __fmul_rn(__int2float_rn((int)r[j]), s4.x);
-            v[j + 1] = __fmul_rn(__int2float_rn((int)r[j + 1]), s4.y);
-            v[j + 2] = __fmul_rn(__int2float_rn((int)r[j + 2]), s4.z);
-            v[j + 3] = __fmul_rn(__int2float_rn((int)r[j + 3]), s4.w);
-        }
-        if (p.bias) {
+            for (int q = 0; q < 8; ++q) {
+                uint32_t x = 0;
 #pragma unroll
-            for (int j = 0; j < 32; j += 4) {
-                const float4 b4 = *reinterpret_cast<const float4*>(bs + j);
-                v[j] = __fadd_rn(v[j], b4.x);
-                v[j + 1] = __fadd_rn(v[j + 1], b4.y);
-                v[j + 2] = __fadd_rn(v[j + 2], b4.z);
-                v[j + 3] = __fadd_rn(v[j + 3], b4.w);
+                for (int i = 0; i < 4; ++i)
+                    if (col0 + 4 * q + i < p.N) x |= (uint32_t)(uint8_t)rp[4 * q + i] << (8 * i);
+                w[q] = x;
             }
+            add_residual(v, w, p.res_scale);
         }
         if (p.y_is_i8) {
             // the next layer's INT8 activations: ReLU, one multiply by fl(1 / out_scale), round half to even, clip
@@ -504,7 +537,9 @@ __device__ __forceinline__ void store_chunk_warp(const ContractionArgs& p, int r
                                                  const CUtensorMap* tmY, const CUtensorMap* tmAcc, const OutCoords& oc) {
     const bool full_chunk = col0 + 32 <= p.N;
     const bool acc_fast = p.acc_out == nullptr || p.acc_tma || (full_chunk && vec_acc);
-    const bool y_fast = p.y == nullptr || p.y_tma || (!p.y_is_i8 && full_chunk && (p.y_is_bf16 ? vec_bf16 : vec_f32));
+    const bool res_fast = p.residual == nullptr ||
+                          (full_chunk && ((p.ld_res & 15) == 0) && ((reinterpret_cast<uintptr_t>(p.residual) & 15) == 0));
+    const bool y_fast = (p.y == nullptr || p.y_tma || (!p.y_is_i8 && full_chunk && (p.y_is_bf16 ? vec_bf16 : vec_f32))) && res_fast;
     if (!acc_fast || !y_fast) {                        // ragged or unaligned: the plain per-row path
         if (row_ok) store_chunk(p, row, col0, r, sc, bs, vec_acc, vec_f32, vec_bf16);
         return;
@@ -523,26 +558,16 @@ __device__ __forceinline__ void store_chunk_warp(const ContractionArgs& p, int r
         }
     }
     if (p.y) {
-        // the 32 factors are the same for every lane: read them four at a time (a scalar read per column costs
-        // a shared-memory wavefront each, and the load/store data path is the busiest unit of this epilogue)
         float v[32];
-#pragma unroll
-        for (int j = 0; j < 32; j += 4) {
-            const float4 s4 = *reinterpret_cast<const float4*>(sc + j);
-            v[j] = __fmul_rn(__int2float_rn((int)r[j]), s4.x);
-            v[j + 1] = __fmul_rn(__int2float_rn((int)r[j + 1]), s4.y);
-            v[j + 2] = __fmul_rn(__int2float_rn((int)r[j + 2]), s4.z);
-            v[j + 3] = __fmul_rn(__int2float_rn((int)r[j + 3]), s4.w);
-        }
-        if (p.bias) {
-#pragma unroll
-            for (int j = 0; j < 32; j += 4) {
-                const float4 b4 = *reinterpret_cast<const float4*>(bs + j);
-                v[j] = __fadd_rn(v[j], b4.x);
-                v[j + 1] = __fadd_rn(v[j + 1], b4.y);
-                v[j + 2] = __fadd_rn(v[j + 2], b4.z);
-                v[j + 3] = __fadd_rn(v[j + 3], b4.w);
+        dequant_chunk(p, r, sc, bs, v);
+        if (p.residual) {                              // a row outside the output adds zeros (its values are clipped by the store)
+            uint4 ra = make_uint4(0u, 0u, 0u, 0u), rb = ra;
+            if (row_ok) {
+                const uint4* rp = reinterpret_cast<const uint4*>(p.residual + (long long)row * p.ld_res + col0);
+                ra = __ldg(rp); rb = __ldg(rp + 1);
             }
+            const uint32_t w[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
+            add_residual(v, w, p.res_scale);
         }
         if (p.y_is_i8) {
             // the next layer's INT8 activations: ReLU, one multiply by fl(1 / out_scale), round half to even, clip
@@ -608,6 +633,123 @@ __device__ __forceinline__ void fetch_scales(const ContractionArgs& p, int col_b
             if (p.bias) bs[i] = __ldg(p.bias + col);
         }
     }
+}
+
+// What an epilogue warp needs from its kernel: where scales, staging blocks and accumulator barriers live, and
+// which tiles the block walks.
+struct EpilogueCtx {
+    float* sScale;
+    float* sBias;
+    uint8_t* sStage;
+    uint64_t* tfull;
+    uint64_t* tempty;
+    uint32_t* signal_sink;        // pair kernel: landing place of signal stores in the leader
+    volatile int* abort_flag;
+    uint32_t tmem_base;
+    int first_tile, tile_step, num_tiles;
+    uint32_t rank;                // pair kernel: this CTA's rank in the pair (0 = leader); 0 otherwise
+};
+
+// The epilogue role of both contraction kernels (warps 2 .. 2 + kEpiWarps - 1): for every tile of the block, wait
+// for the accumulator, read this warp's lane quarter and half of the columns 32 columns at a time, hand the
+// accumulator back after the last read, dequantise and store.  BN: tile columns.  PAIR: the block is one CTA of a
+// pair -- it owns rows [128 * rank, 128 * rank + 128) of a 256-row tile, the accumulator barriers are signalled
+// across the pair (tfull by the leader's commit in both CTAs; tempty lives in the leader, to which the partner's
+// warps send 4 announced bytes each).
+template <int BN, int MODE, bool PAIR>
+__device__ __forceinline__ void epilogue_role(const ContractionArgs& p, const CUtensorMap* tmY, const CUtensorMap* tmAcc,
+                                              const EpilogueCtx& ex, int warp, int lane) {
+    using namespace sm100;
+    const int quarter = warp & 3;                  // TMEM lanes this warp may read
+    const int chalf = (warp - 2) >> 2;             // which half of the tile's columns it handles
+    int staged_nt = -1;                            // column tile whose scales sit in shared memory
+    constexpr int SCALES_PER_LANE = BN / 64;       // a warp stages BN / 2 scales
+    uint32_t tl = 0;
+    bool ok = true;
+    const bool vec_f32 = (p.y != nullptr) && !p.y_is_bf16 && ((p.ldy & 3) == 0) &&
+                         ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
+    const bool vec_bf16 = (p.y != nullptr) && p.y_is_bf16 && ((p.ldy & 7) == 0) &&
+                          ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
+    const bool vec_acc = (p.acc_out != nullptr) && ((p.ld_acc & 3) == 0) &&
+                         ((reinterpret_cast<uintptr_t>(p.acc_out) & 15) == 0);
+    // per-channel factor: fl(fl(act * w_scale) * 2^l), then the exact 2^-(8-h) of the unpack.
+    // Each warp keeps a private copy, so the epilogue warps never wait on one another.
+    float* sc_w = ex.sScale + (warp - 2) * (BN / 2);      // scales of this warp's half of the columns
+    float* bs_w = ex.sBias + (warp - 2) * (BN / 2);
+    for (int tile = ex.first_tile; ok && tile < ex.num_tiles; tile += ex.tile_step, ++tl) {
+        int mt, nt;
+        tile_coords(tile, p, mt, nt);
+        if (PAIR) mt = mt * 2 + (int)ex.rank;          // this CTA's 128-row tile of the pair's 256 rows
+        const uint32_t buf = tl & 1, buse = tl >> 1;
+        const int n0 = nt * BN;
+        __syncwarp();
+        if (nt != staged_nt) {                         // only the first tile: later ones are prefetched below
+            float sc_r[SCALES_PER_LANE], bs_r[SCALES_PER_LANE];
+            fetch_scales<SCALES_PER_LANE>(p, n0 + chalf * (BN / 2), lane, sc_r, bs_r);
+#pragma unroll
+            for (int i = 0; i < SCALES_PER_LANE; ++i) { sc_w[lane + 32 * i] = sc_r[i]; bs_w[lane + 32 * i] = bs_r[i]; }
+            staged_nt = nt;
+        }
+        __syncwarp();
+        // The next tile's scales are fetched now and land in registers while this tile is converted and
+        // stored; they go to shared memory at the end of the iteration.  (Fetched at the top of the next
+        // iteration instead, the global-memory round trip sat on every tile's critical path.)
+        int next_nt = -1;
+        float sc_n[SCALES_PER_LANE], bs_n[SCALES_PER_LANE];
+        if (tile + ex.tile_step < ex.num_tiles) {
+            int mt_n;
+            tile_coords(tile + ex.tile_step, p, mt_n, next_nt);
+            if (next_nt != nt) fetch_scales<SCALES_PER_LANE>(p, next_nt * BN + chalf * (BN / 2), lane, sc_n, bs_n);
+        }
+        ok = PAIR ? mbar_wait_cluster(smem_u32(&ex.tfull[buf]), buse & 1, ex.abort_flag, p.status, 0x130u)
+                  : mbar_wait(smem_u32(&ex.tfull[buf]), buse & 1, ex.abort_flag, p.status, 0x30u);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after_sync();
+        long long row;
+        bool row_ok;
+        if (MODE == kModeGemm) {
+            row = (long long)mt * kBM + quarter * 32 + lane;
+            row_ok = row < p.M;
+        } else {
+            // tile row -> output pixel: the low bits walk the width, then the height, then the images
+            const TileOrigin o = conv_tile_origin(p.g, mt);
+            const int ml = quarter * 32 + lane;
+            const int qq = o.q0 + (ml & ((1 << p.g.tw_log2) - 1));
+            const int pp = o.p0 + ((ml >> p.g.tw_log2) & ((1 << p.g.th_log2) - 1));
+            const int bb = o.b0 + (ml >> (p.g.tw_log2 + p.g.th_log2));
+            row_ok = qq < p.g.Wo && pp < p.g.Ho && bb < p.g.B;
+            row = ((long long)bb * p.g.Ho + pp) * p.g.Wo + qq;
+        }
+        const OutCoords oc = out_coords<MODE>(p, mt, quarter * 32);
+        constexpr int CHUNKS = BN / 64;                // 32-column chunks per warp (half of the tile)
+#pragma unroll 1
+        for (int cc = 0; cc < CHUNKS; ++cc) {
+            const int c = chalf * CHUNKS + cc;
+            uint32_t r[32];
+            tmem_ld_32x32(ex.tmem_base + buf * BN + c * 32 + ((uint32_t)(quarter * 32) << 16), r);
+            tmem_ld_wait();
+            if (cc == CHUNKS - 1) {                    // last read of the accumulator: hand it back before storing
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) {
+                    if (!PAIR || ex.rank == 0) mbar_arrive(smem_u32(&ex.tempty[buf]));
+                    else signal_remote_tx4(map_to_cta(smem_u32(ex.signal_sink), 0), map_to_cta(smem_u32(&ex.tempty[buf]), 0));
+                }
+            }
+            const int col0 = n0 + c * 32;
+            if (col0 >= p.N) continue;
+            store_chunk_warp(p, (int)row, row_ok, col0, r, sc_w + cc * 32, bs_w + cc * 32, vec_acc, vec_f32, vec_bf16,
+                             ex.sStage + (warp - 2) * kEpiStageBytes, lane, tmY, tmAcc, oc);
+        }
+        if (next_nt >= 0 && next_nt != nt) {
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < SCALES_PER_LANE; ++i) { sc_w[lane + 32 * i] = sc_n[i]; bs_w[lane + 32 * i] = bs_n[i]; }
+            staged_nt = next_nt;
+        }
+    }
+    if (lane == 0) bulk_wait_all();                    // this lane's tile stores are done before the block leaves
 }
 
 // Part-bit blocks end with one more warp, the producer of the packed-tile ring: two producers that spin in one
@@ -787,91 +929,11 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         }
     } else if (warp < kFirstUnpackWarp) {
         // ------------------------------------------------------------------ epilogue
-        const int quarter = warp & 3;                  // TMEM lanes this warp may read
-        const int chalf = (warp - 2) >> 2;             // which half of the tile's columns it handles
-        int staged_nt = -1;                            // column tile whose scales sit in shared memory
-        constexpr int SCALES_PER_LANE = BN / 64;       // a warp stages BN / 2 scales
-        uint32_t tl = 0;
-        bool ok = true;
-        const bool vec_f32 = (p.y != nullptr) && !p.y_is_bf16 && ((p.ldy & 3) == 0) &&
-                             ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
-        const bool vec_bf16 = (p.y != nullptr) && p.y_is_bf16 && ((p.ldy & 7) == 0) &&
-                              ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
-        const bool vec_acc = (p.acc_out != nullptr) && ((p.ld_acc & 3) == 0) &&
-                             ((reinterpret_cast<uintptr_t>(p.acc_out) & 15) == 0);
-        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++tl) {
-            int mt, nt;
-            tile_coords(tile, p, mt, nt);
-            const uint32_t buf = tl & 1, buse = tl >> 1;
-            const int n0 = nt * BN;
-            // per-channel factor: fl(fl(act * w_scale) * 2^l), then the exact 2^-(8-h) of the unpack.
-            // Each warp keeps a private copy, so the epilogue warps never wait on one another.
-            float* sc_w = sScale + (warp - 2) * (BN / 2);      // scales of this warp's half of the columns
-            float* bs_w = sBias + (warp - 2) * (BN / 2);
-            __syncwarp();
-            if (nt != staged_nt) {                         // only the first tile: later ones are prefetched below
-                float sc_r[SCALES_PER_LANE], bs_r[SCALES_PER_LANE];
-                fetch_scales<SCALES_PER_LANE>(p, n0 + chalf * (BN / 2), lane, sc_r, bs_r);
-#pragma unroll
-                for (int i = 0; i < SCALES_PER_LANE; ++i) { sc_w[lane + 32 * i] = sc_r[i]; bs_w[lane + 32 * i] = bs_r[i]; }
-                staged_nt = nt;
-            }
-            __syncwarp();
-            // The next tile's scales are fetched now and land in registers while this tile is converted and
-            // stored; they go to shared memory at the end of the iteration.  (Fetched at the top of the next
-            // iteration instead, the global-memory round trip sat on every tile's critical path.)
-            int next_nt = -1;
-            float sc_n[SCALES_PER_LANE], bs_n[SCALES_PER_LANE];
-            if (tile + (int)gridDim.x < num_tiles) {
-                int mt_n;
-                tile_coords(tile + (int)gridDim.x, p, mt_n, next_nt);
-                if (next_nt != nt) fetch_scales<SCALES_PER_LANE>(p, next_nt * BN + chalf * (BN / 2), lane, sc_n, bs_n);
-            }
-            ok = mbar_wait(smem_u32(&tfull[buf]), buse & 1, abort_flag, p.status, 0x30u);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after_sync();
-            long long row;
-            bool row_ok;
-            if (MODE == kModeGemm) {
-                row = (long long)mt * kBM + quarter * 32 + lane;
-                row_ok = row < p.M;
-            } else {
-                // tile row -> output pixel: the low bits walk the width, then the height, then the images
-                const TileOrigin o = conv_tile_origin(p.g, mt);
-                const int ml = quarter * 32 + lane;
-                const int qq = o.q0 + (ml & ((1 << p.g.tw_log2) - 1));
-                const int pp = o.p0 + ((ml >> p.g.tw_log2) & ((1 << p.g.th_log2) - 1));
-                const int bb = o.b0 + (ml >> (p.g.tw_log2 + p.g.th_log2));
-                row_ok = qq < p.g.Wo && pp < p.g.Ho && bb < p.g.B;
-                row = ((long long)bb * p.g.Ho + pp) * p.g.Wo + qq;
-            }
-            const OutCoords oc = out_coords<MODE>(p, mt, quarter * 32);
-            constexpr int CHUNKS = BN / 64;                // 32-column chunks per warp (half of the tile)
-#pragma unroll 1
-            for (int cc = 0; cc < CHUNKS; ++cc) {
-                const int c = chalf * CHUNKS + cc;
-                uint32_t r[32];
-                tmem_ld_32x32(tmem_base + buf * BN + c * 32 + ((uint32_t)(quarter * 32) << 16), r);
-                tmem_ld_wait();
-                if (cc == CHUNKS - 1) {                    // last read of the accumulator: hand it back before storing
-                    tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&tempty[buf]));
-                }
-                const int col0 = n0 + c * 32;
-                if (col0 >= p.N) continue;
-                store_chunk_warp(p, (int)row, row_ok, col0, r, sc_w + cc * 32, bs_w + cc * 32, vec_acc, vec_f32, vec_bf16,
-                                 sStage + (warp - 2) * kEpiStageBytes, lane, &tmY, &tmAcc, oc);
-            }
-            if (next_nt >= 0 && next_nt != nt) {
-                __syncwarp();
-#pragma unroll
-                for (int i = 0; i < SCALES_PER_LANE; ++i) { sc_w[lane + 32 * i] = sc_n[i]; bs_w[lane + 32 * i] = bs_n[i]; }
-                staged_nt = next_nt;
-            }
-        }
-        if (lane == 0) bulk_wait_all();                    // this lane's tile stores are done before the block leaves
+        EpilogueCtx ex;
+        ex.sScale = sScale; ex.sBias = sBias; ex.sStage = sStage; ex.tfull = tfull; ex.tempty = tempty;
+        ex.signal_sink = nullptr; ex.abort_flag = abort_flag; ex.tmem_base = tmem_base;
+        ex.first_tile = blockIdx.x; ex.tile_step = gridDim.x; ex.num_tiles = num_tiles; ex.rank = 0;
+        epilogue_role<BN, MODE, false>(p, &tmY, &tmAcc, ex, warp, lane);
     } else if (PART && warp < kPackedProducerWarp) {
         // ------------------------------------------------------------------ unpackers
         const int utid = threadIdx.x - kBaseThreads;
@@ -920,6 +982,8 @@ constexpr int kOutI8 = 2;
 struct OutQuant {
     float out_scale;
     int relu;
+    const int8_t* residual;   // INT8 skip tensor of the output's shape (dense), or nullptr
+    float res_scale;
 };
 
 // Host launcher (defined with the GEMM entry points).  The A operand is reached through tmA: a plain 2-D map

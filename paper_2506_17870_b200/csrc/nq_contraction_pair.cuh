@@ -388,92 +388,11 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         }
     } else if (warp < kFirstUnpackWarp) {
         // ------------------------------------------------------------------ epilogue (both CTAs, own 128 rows)
-        const int quarter = warp & 3;
-        const int chalf = (warp - 2) >> 2;             // which half of the tile's columns this warp handles
-        int staged_nt = -1;                            // column tile whose scales sit in shared memory
-        constexpr int SCALES_PER_LANE = BN / 64;       // a warp stages BN / 2 scales
-        uint32_t tl = 0;
-        bool ok = true;
-        const bool vec_f32 = (p.y != nullptr) && !p.y_is_bf16 && ((p.ldy & 3) == 0) &&
-                             ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
-        const bool vec_bf16 = (p.y != nullptr) && p.y_is_bf16 && ((p.ldy & 7) == 0) &&
-                              ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
-        const bool vec_acc = (p.acc_out != nullptr) && ((p.ld_acc & 3) == 0) &&
-                             ((reinterpret_cast<uintptr_t>(p.acc_out) & 15) == 0);
-        float* sc_w = sScale + (warp - 2) * (BN / 2);      // scales of this warp's half of the columns
-        float* bs_w = sBias + (warp - 2) * (BN / 2);
-        for (int tile = pair; ok && tile < num_tiles; tile += num_pairs, ++tl) {
-            int mt2, nt;
-            tile_coords(tile, p, mt2, nt);
-            const int mt = mt2 * 2 + (int)rank;
-            const uint32_t buf = tl & 1, buse = tl >> 1;
-            const int n0 = nt * BN;
-            __syncwarp();
-            if (nt != staged_nt) {                         // only the first tile: later ones are prefetched below
-                float sc_r[SCALES_PER_LANE], bs_r[SCALES_PER_LANE];
-                fetch_scales<SCALES_PER_LANE>(p, n0 + chalf * (BN / 2), lane, sc_r, bs_r);
-#pragma unroll
-                for (int i = 0; i < SCALES_PER_LANE; ++i) { sc_w[lane + 32 * i] = sc_r[i]; bs_w[lane + 32 * i] = bs_r[i]; }
-                staged_nt = nt;
-            }
-            __syncwarp();
-            // The next tile's scales are fetched now and land in registers while this tile is converted and
-            // stored; they go to shared memory at the end of the iteration.  (Fetched at the top of the next
-            // iteration instead, the global-memory round trip sat on every tile's critical path.)
-            int next_nt = -1;
-            float sc_n[SCALES_PER_LANE], bs_n[SCALES_PER_LANE];
-            if (tile + num_pairs < num_tiles) {
-                int mt_n;
-                tile_coords(tile + num_pairs, p, mt_n, next_nt);
-                if (next_nt != nt) fetch_scales<SCALES_PER_LANE>(p, next_nt * BN + chalf * (BN / 2), lane, sc_n, bs_n);
-            }
-            ok = mbar_wait_cluster(smem_u32(&tfull[buf]), buse & 1, abort_flag, p.status, 0x130u);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after_sync();
-            long long row;
-            bool row_ok;
-            if (MODE == kModeGemm) {
-                row = (long long)mt * kBM + quarter * 32 + lane;
-                row_ok = row < p.M;
-            } else {
-                const TileOrigin o = conv_tile_origin(p.g, mt);
-                const int ml = quarter * 32 + lane;
-                const int qq = o.q0 + (ml & ((1 << p.g.tw_log2) - 1));
-                const int pp = o.p0 + ((ml >> p.g.tw_log2) & ((1 << p.g.th_log2) - 1));
-                const int bb = o.b0 + (ml >> (p.g.tw_log2 + p.g.th_log2));
-                row_ok = qq < p.g.Wo && pp < p.g.Ho && bb < p.g.B;
-                row = ((long long)bb * p.g.Ho + pp) * p.g.Wo + qq;
-            }
-            const OutCoords oc = out_coords<MODE>(p, mt, quarter * 32);
-            constexpr int CHUNKS = BN / 64;                // 32-column chunks per warp (half of the tile)
-#pragma unroll 1
-            for (int cc = 0; cc < CHUNKS; ++cc) {
-                const int c = chalf * CHUNKS + cc;
-                uint32_t r[32];
-                tmem_ld_32x32(tmem_base + buf * BN + c * 32 + ((uint32_t)(quarter * 32) << 16), r);
-                tmem_ld_wait();
-                if (cc == CHUNKS - 1) {                    // last read of the accumulator: hand it back before storing
-                    tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) {
-                        if (rank == 0) mbar_arrive(smem_u32(&tempty[buf]));
-                        else signal_remote_tx4(map_to_cta(smem_u32(signal_sink), 0), map_to_cta(smem_u32(&tempty[buf]), 0));
-                    }
-                }
-                const int col0 = n0 + c * 32;
-                if (col0 >= p.N) continue;
-                store_chunk_warp(p, (int)row, row_ok, col0, r, sc_w + cc * 32, bs_w + cc * 32, vec_acc, vec_f32, vec_bf16,
-                                 sStage + (warp - 2) * kEpiStageBytes, lane, &tmY, &tmAcc, oc);
-            }
-            if (next_nt >= 0 && next_nt != nt) {
-                __syncwarp();
-#pragma unroll
-                for (int i = 0; i < SCALES_PER_LANE; ++i) { sc_w[lane + 32 * i] = sc_n[i]; bs_w[lane + 32 * i] = bs_n[i]; }
-                staged_nt = next_nt;
-            }
-        }
-        if (lane == 0) bulk_wait_all();                    // this lane's tile stores are done before the block leaves
+        EpilogueCtx ex;
+        ex.sScale = sScale; ex.sBias = sBias; ex.sStage = sStage; ex.tfull = tfull; ex.tempty = tempty;
+        ex.signal_sink = signal_sink; ex.abort_flag = abort_flag; ex.tmem_base = tmem_base;
+        ex.first_tile = pair; ex.tile_step = num_pairs; ex.num_tiles = num_tiles; ex.rank = rank;
+        epilogue_role<BN, MODE, true>(p, &tmY, &tmAcc, ex, warp, lane);
     } else if (PART && DIRECT) {
         // ------------------------------------------------------------------ unpackers reading global memory (h <= 4)
         PairUnpackCtx cx;

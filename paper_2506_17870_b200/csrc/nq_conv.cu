@@ -331,6 +331,26 @@ int nq_conv_implicit_gemm_q8(const int8_t* X, const void* Wt, int64_t ldw, int p
                        workspace_bytes, stream, &oq);
 }
 
+int nq_conv_implicit_gemm_q8_res(const int8_t* X, const void* Wt, int64_t ldw, int part_bit, int n_bits, int h_bits,
+                                 const nq_conv_desc* d, const float* w_scale, float act_scale, const float* bias,
+                                 const int8_t* residual, float residual_scale, float out_scale, int relu, int8_t* Yq,
+                                 void* workspace, int64_t workspace_bytes, void* stream) {
+    const nq::OutQuant oq{out_scale, relu, residual, residual_scale};
+    if (!Yq || !residual) return NQ_ERR_INVALID_ARG;
+    return conv_common(X, Wt, ldw, part_bit, n_bits, h_bits, d, w_scale, act_scale, bias, nullptr, Yq, nq::kOutI8, workspace,
+                       workspace_bytes, stream, &oq);
+}
+
+int nq_conv_implicit_gemm_nested_q8_res(const int8_t* X, const void* packed_high, const void* packed_low, int n_bits,
+                                        int h_bits, const nq_conv_desc* d, const float* w_scale, float act_scale,
+                                        const float* bias, const int8_t* residual, float residual_scale, float out_scale,
+                                        int relu, int8_t* Yq, void* workspace, int64_t workspace_bytes, void* stream) {
+    const nq::OutQuant oq{out_scale, relu, residual, residual_scale};
+    if (!Yq || !packed_low || !residual) return NQ_ERR_INVALID_ARG;
+    return conv_common(X, packed_high, 0, 1, n_bits, h_bits, d, w_scale, act_scale, bias, nullptr, Yq, nq::kOutI8, workspace,
+                       workspace_bytes, stream, &oq, packed_low);
+}
+
 int nq_conv_implicit_gemm_static(const int8_t* X, const void* Wt, int64_t ldw, int part_bit, int n_bits, int h_bits,
                                  const nq_conv_desc* d, const float* w_scale, float act_scale, const float* bias,
                                  int32_t* acc_out, void* Y, int y_dtype, void* stream) {

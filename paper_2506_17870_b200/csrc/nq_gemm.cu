@@ -4,7 +4,6 @@
 #include <stdint.h>
 
 #include "../../include/nq.h"
-#include <stdlib.h>
 
 #include "nq_contraction_pair.cuh"
 #include "nq_internal.cuh"
@@ -154,11 +153,11 @@ int launch_pair_mode(int mode, const CUtensorMap& tmA, const CUtensorMap& tmB, c
     return launch_pair<PART, kModeGemm, DIRECT>(tmA, tmB, om, a, s);
 }
 
-// NQ_PLAIN_STORES=1 in the environment keeps the epilogue on ordinary global stores (for comparisons and tests)
-bool tile_stores_enabled() {
-    const char* e = getenv("NQ_PLAIN_STORES");
-    return !(e && e[0] == '1');
-}
+// Test switches (nq_debug_set): keep the epilogue on ordinary global stores / keep every part-bit pair launch on the
+// TMA-fed ring of packed tiles, so that tests can compare those paths with the default ones bit for bit.
+int g_debug[2] = {0, 0};
+bool tile_stores_enabled() { return g_debug[NQ_DEBUG_PLAIN_STORES] == 0; }
+bool direct_fetch_enabled() { return g_debug[NQ_DEBUG_PACKED_RING] == 0; }
 
 // Tile-store map of one output ([M, N] of esize-byte elements, pitch ld): possible when base and pitch are
 // 16-byte aligned.  Convolution outputs are NHWC, addressed by (pixel column, pixel row, image) in boxes that
@@ -175,23 +174,6 @@ bool make_out_map(CUtensorMap* map, const void* base, int esize, int64_t M, int6
     const uint32_t bb = 32 / (bw * bh);
     return encode_tensor_map_out(map, base, row_bytes, pitch, (uint64_t)g->Wo, (uint64_t)g->Ho, (uint64_t)g->B, bw, bh, bb,
                                  box_bytes) == NQ_OK;
-}
-
-// NQ_PACKED_RING=1 in the environment keeps every part-bit pair launch on the TMA-fed ring of packed tiles
-// (for comparisons and tests); otherwise h = 1, 2, 4 read the packed matrix directly (nq_contraction_pair.cuh).
-bool direct_fetch_enabled() {
-    const char* e = getenv("NQ_PACKED_RING");
-    return !(e && e[0] == '1');
-}
-
-// NQ_SINGLE_CTA=1 in the environment keeps every contraction on the one-CTA-per-tile kernel (for comparisons)
-bool pairs_enabled() {
-    static int cached = -1;
-    if (cached < 0) {
-        const char* e = getenv("NQ_SINGLE_CTA");
-        cached = (e && e[0] == '1') ? 0 : 1;
-    }
-    return cached == 1;
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
@@ -224,7 +206,7 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
         const double stage_cycles[4] = {260.0, 330.0, 800.0, 560.0};
         for (int c = 0; c < 4; ++c) {
             if (nest && !cand_pair[c]) continue;
-            if (cand_pair[c] && !nest && (!pairs_enabled() || m_tiles < 2)) continue;
+            if (cand_pair[c] && !nest && m_tiles < 2) continue;
             if (c > 0 && N <= cand_bn[c - 1] && !(c == 3)) continue;          // no wider than the output needs
             if (c == 3 && N <= 128 && !nest) continue;
             const long long nt = (N + cand_bn[c] - 1) / cand_bn[c];
@@ -249,6 +231,9 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
     a.y_is_i8 = (y_dtype == kOutI8 && oq) ? 1 : 0;
     a.relu = oq ? oq->relu : 0;
     a.inv_out_scale = oq ? 1.0f / oq->out_scale : 1.0f;
+    a.residual = (oq && a.y_is_i8) ? oq->residual : nullptr;      // dense, like the output
+    a.ld_res = N;
+    a.res_scale = oq ? oq->res_scale : 0.0f;
     a.status = status_word();
     if (!a.status) return NQ_ERR_CUDA;
     OutMaps om;
@@ -361,6 +346,12 @@ int gemm_common(const int8_t* X, int64_t ldx, const void* Bmat, int64_t ldb, boo
 }  // namespace nq
 
 extern "C" {
+
+int nq_debug_set(int which, int enabled) {
+    if (which != NQ_DEBUG_PLAIN_STORES && which != NQ_DEBUG_PACKED_RING) return NQ_ERR_INVALID_ARG;
+    nq::g_debug[which] = enabled ? 1 : 0;
+    return NQ_OK;
+}
 
 int nq_gemm_full(const int8_t* X, int64_t ldx, const int8_t* W, int64_t ldw, const float* w_scale, float act_scale,
                  const float* bias, int64_t M, int64_t N, int64_t K, int32_t* acc_out, int64_t ld_acc, void* Y,

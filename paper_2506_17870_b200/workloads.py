@@ -203,3 +203,49 @@ def oihw_to_ohwi_matrix(w_oihw: np.ndarray, ld: int = 0) -> np.ndarray:
         out[:, : m.shape[1]] = m
         return out
     return m
+
+
+# --------------------------------------------------------------------------- dependent chains (structure only)
+def resnet_chain_plan(layers: List[ConvLayer]) -> List[Dict[str, object]]:
+    """A ResNet-shaped layer table as ONE dependent chain: which tensor every layer reads and writes.  Pure
+    structure (no arithmetic): stem -> 3x3 / 2 max pooling -> residual blocks (basic blocks c1, c2 or bottlenecks
+    c1, c2, c3; the last convolution of a block adds the skip tensor -- the block's input, or its 1x1 down-sampling
+    convolution `ds` -- before the ReLU) -> global average pooling -> classifier.  Steps:
+      {"op": "conv", "layer": name, "src": tensor, "dst": tensor, "relu": bool, "skip": tensor or None}
+      {"op": "maxpool", "src", "dst", "k", "stride", "pad"},  {"op": "avgpool", "src", "dst"},
+      {"op": "fc", "layer": "fc", "src", "dst"}                      (fp32 logits, no requantisation)"""
+    by = {L.name: L for L in layers}
+    steps: List[Dict[str, object]] = [
+        {"op": "conv", "layer": "conv1", "src": "input", "dst": "stem", "relu": True, "skip": None},
+        {"op": "maxpool", "src": "stem", "dst": "pool", "k": 3, "stride": 2, "pad": 1},
+    ]
+    cur = "pool"
+    for stage in range(1, 5):
+        block = 0
+        while f"l{stage}b{block}c1" in by:
+            pre = f"l{stage}b{block}"
+            convs = [c for c in ("c1", "c2", "c3") if pre + c in by]
+            skip = cur
+            if pre + "ds" in by:
+                steps.append({"op": "conv", "layer": pre + "ds", "src": cur, "dst": pre + "ds", "relu": False, "skip": None})
+                skip = pre + "ds"
+            t = cur
+            for c in convs[:-1]:
+                steps.append({"op": "conv", "layer": pre + c, "src": t, "dst": pre + c, "relu": True, "skip": None})
+                t = pre + c
+            steps.append({"op": "conv", "layer": pre + convs[-1], "src": t, "dst": pre + "out", "relu": True, "skip": skip})
+            cur = pre + "out"
+            block += 1
+    steps.append({"op": "avgpool", "src": cur, "dst": "pooled"})
+    steps.append({"op": "fc", "layer": "fc", "src": "pooled", "dst": "logits"})
+    return steps
+
+
+def chain_weights(config: int, layers: List[ConvLayer]) -> Dict[str, Dict[str, np.ndarray]]:
+    """Seeded weights of every layer of a chain: Gaussian fit + per-channel INT8 (OIHW), scales, rounding mask."""
+    out = {}
+    for i, L in enumerate(layers):
+        rng = rng_for(config, 500 + i)
+        w, s = gaussian_weights_int8(rng, (L.Cout, L.Cin, L.R, L.S), L.K)
+        out[L.name] = {"W": w, "w_scale": s, "mask": bernoulli_mask(rng, w.shape)}
+    return out

@@ -24,3 +24,18 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture
+def debug_switch():
+    """Turns one of the library's test switches (nq_debug_set) on for the rest of a test and off again afterwards."""
+    import paper_2506_17870_b200 as nq
+    used = []
+
+    def on(which):
+        nq.nq_debug_set(which, True)
+        used.append(which)
+
+    yield on
+    for which in used:
+        nq.nq_debug_set(which, False)

@@ -98,7 +98,7 @@ def test_other_nestings(h):
 
 @pytest.mark.parametrize("L", [C("c64_wide", 64, 40, 40, 64, 3, 3, 1, 1), C("c128_ragged", 128, 13, 9, 72, 3, 3, 2, 1)],
                          ids=lambda l: l.name)
-def test_tile_stores_and_plain_stores_agree(L, monkeypatch):
+def test_tile_stores_and_plain_stores_agree(L, debug_switch):
     """NHWC outputs go out as 4-D tile stores whose boxes follow the pixel rectangle of a tile (pixels outside the
     image are clipped by the store); the ordinary-store epilogue must give the same bytes."""
     run_layer(L, 3, 77)
@@ -108,7 +108,7 @@ def test_tile_stores_and_plain_stores_agree(L, monkeypatch):
     desc = nq.nq_conv_desc(3, L.Cin, L.H, L.W, L.Cout, L.R, L.S, L.stride, L.pad, 1)
     x, ws = dev(d["X"]), dev(d["w_scale"])
     acc, y, _ = nq.nq_conv_implicit_gemm(x, w_mat, desc, ws, 0.02, want_acc=True, y_dtype=torch.bfloat16)
-    monkeypatch.setenv("NQ_PLAIN_STORES", "1")
+    debug_switch(nq.NQ_DEBUG_PLAIN_STORES)
     acc2, y2, _ = nq.nq_conv_implicit_gemm(x, w_mat, desc, ws, 0.02, want_acc=True, y_dtype=torch.bfloat16)
     nq.nq_device_status()
     assert torch.equal(acc, acc2) and torch.equal(y.view(torch.int16), y2.view(torch.int16))

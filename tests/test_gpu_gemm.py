@@ -130,7 +130,7 @@ def test_full_equals_shifted_part_plus_low_contribution():
 
 
 @pytest.mark.parametrize("h", [1, 2, 3, 4, 5, 6, 7])
-def test_wide_ragged_gemm_narrow_fields(h, monkeypatch):
+def test_wide_ragged_gemm_narrow_fields(h, debug_switch):
     """Large enough for the CTA-pair kernel, whose unpack warps read fields of 1, 2 and 4 bits straight from the
     packed matrix: ragged in M, N and K, every width checked against the oracle, and bit for bit against the same
     launch with every width fed through the shared-memory ring of packed tiles."""
@@ -142,7 +142,7 @@ def test_wide_ragged_gemm_narrow_fields(h, monkeypatch):
     acc, y = nq.nq_gemm_part(Xd, hi, N, 8, h, wsd, d["act_scale"], want_acc=True)
     nq.nq_device_status()
     check_outputs(acc, y, oracle.gemm_acc(d["X"], wh), d["w_scale"], d["act_scale"], 8 - h)
-    monkeypatch.setenv("NQ_PACKED_RING", "1")
+    debug_switch(nq.NQ_DEBUG_PACKED_RING)
     acc2, y2 = nq.nq_gemm_part(Xd, hi, N, 8, h, wsd, d["act_scale"], want_acc=True)
     nq.nq_device_status()
     assert torch.equal(acc, acc2) and torch.equal(y, y2)
@@ -150,7 +150,7 @@ def test_wide_ragged_gemm_narrow_fields(h, monkeypatch):
 
 @pytest.mark.parametrize("M,N,K,bf16", [(300, 520, 1000, False), (300, 520, 1000, True), (1030, 1100, 640, True),
                                          (130, 40, 147, False), (2100, 72, 256, True)])
-def test_tile_stores_and_plain_stores_agree(M, N, K, bf16, monkeypatch):
+def test_tile_stores_and_plain_stores_agree(M, N, K, bf16, debug_switch):
     """The epilogue writes aligned outputs with TMA tile stores (ragged rows and columns clipped by the store) and
     everything else with ordinary stores: both against the oracle, and bit for bit against each other."""
     d = wl.gemm_inputs(90, M + N + K, M, N, K)
@@ -159,7 +159,7 @@ def test_tile_stores_and_plain_stores_agree(M, N, K, bf16, monkeypatch):
     Xd, wsd = dev_padded(d["X"]), dev(d["w_scale"])
     ydt = torch.bfloat16 if bf16 else torch.float32
     acc, y = nq.nq_gemm_part(Xd, hi, N, 8, 6, wsd, d["act_scale"], want_acc=True, y_dtype=ydt)
-    monkeypatch.setenv("NQ_PLAIN_STORES", "1")
+    debug_switch(nq.NQ_DEBUG_PLAIN_STORES)
     acc2, y2 = nq.nq_gemm_part(Xd, hi, N, 8, 6, wsd, d["act_scale"], want_acc=True, y_dtype=ydt)
     nq.nq_device_status()
     assert torch.equal(acc, acc2) and torch.equal(y.view(torch.int16 if bf16 else torch.int32),
