@@ -23,14 +23,19 @@
  *     for n_bits < 8 values outside [-2^(n-1), 2^(n-1) - 1] give unspecified results.
  *
  * Packed ("sliced") layout of a [rows, cols] tensor of k-bit two's-complement fields
- *   Each row is padded with zero fields to a multiple of 128 and cut into groups of 128 elements;
- *   a group is 16*k bytes, a row nq_packed_row_bytes(cols, k) bytes, rows follow one another.
- *   k is split into powers of two (8, 4, 2, 1), widest first; the slice of width s holds s bits of
- *   every field (the widest slice the most significant bits) in 16*s bytes.  In a slice, element e
- *   of the group lives in byte ((e/32)*s + ((e%32)/4) / (8/s)) * 4 + e%4, at bits
- *   [8 - s*(sub+1), 8 - s*sub) with sub = ((e%32)/4) % (8/s).  (The paper only fixes the field
- *   width and its two's-complement content; this placement lets four fields be extracted with one
- *   mask per 32-bit word.)  The base address of a packed tensor must be 16-byte aligned.
+ *   The tensor is padded with zero fields to multiples of 128 rows and 128 columns and cut into blocks of
+ *   128 rows x 128 columns.  A block is 2048*k contiguous bytes; block (rb, g) -- row block rb, column group g
+ *   of G = ceil(cols / 128) -- is block number rb*G + g.  The whole tensor takes nq_packed_bytes(rows, cols, k)
+ *   = (rows padded to 128) * nq_packed_row_bytes(cols, k) bytes.
+ *   k is split into powers of two (8, 4, 2, 1), widest first; the slice of width s holds s bits of every field
+ *   (the widest slice the most significant bits) and takes 2048*s bytes of the block: the block's 128 rows one
+ *   after the other, 16*s bytes each.  In a row's 16*s bytes, element e (= column % 128) lives in byte
+ *   ((e/32)*s + ((e%32)/4) / (8/s)) * 4 + e%4, at bits [8 - s*(sub+1), 8 - s*sub) with sub = ((e%32)/4) % (8/s).
+ *   (The paper only fixes the field width and its two's-complement content.  This placement lets four fields be
+ *   extracted with one mask per 32-bit word, and makes the 128 rows x 128 columns that one thread block of the
+ *   GEMM consumes per step one contiguous run of memory.)  The base address of a packed tensor must be 16-byte
+ *   aligned.  Kernels that write a packed tensor write its padding as zero fields; kernels that read one never
+ *   depend on the padding's content.
  */
 #ifndef NQ_H_
 #define NQ_H_
@@ -66,7 +71,8 @@ NQ_API const char *nq_status_str(int status);
 /* Bits of the stored low field: l + 1 with compensation, l without.  Returns -1 for a bad (n, h). */
 NQ_API int nq_low_bits(int n_bits, int h_bits, int compensate);
 
-/* Size of one packed row / of a whole packed tensor in bytes (host, pure).  -1 on bad arguments. */
+/* Bytes per row of the padded tensor (a size unit: 16 * bits per 128 columns; a row's bytes are not contiguous) and
+ * size of a whole packed tensor in bytes, rows padded to a multiple of 128 (host, pure).  -1 on bad arguments. */
 NQ_API int64_t nq_packed_row_bytes(int64_t cols, int bits);
 NQ_API int64_t nq_packed_bytes(int64_t rows, int64_t cols, int bits);
 

@@ -134,23 +134,28 @@ def unpack_word64(words, cols: int, bits: int):
 
 
 def sliced_row_bytes(cols: int, bits: int) -> int:
+    """Bytes per row of a packed tensor (a size unit: the tensor is stored in 128 x 128 blocks)."""
     return int(_load().nqo_sliced_row_bytes(_i64(cols), bits))
 
 
+def sliced_padded_rows(rows: int) -> int:
+    return -(-int(rows) // 128) * 128
+
+
 def pack_sliced(v, bits: int):
+    """-> uint8 [rows padded to 128, sliced_row_bytes(cols, bits)]: the packed tensor's bytes in storage order."""
     v = _c(v, np.int8)
     rows, cols = v.shape
-    out = np.empty((rows, sliced_row_bytes(cols, bits)), dtype=np.uint8)
+    out = np.empty((sliced_padded_rows(rows), sliced_row_bytes(cols, bits)), dtype=np.uint8)
     rc = _load().nqo_pack_sliced(_p(v), _i64(rows), _i64(cols), bits, _p(out))
     if rc != 0:
         raise ValueError("unsupported field width")
     return out
 
 
-def unpack_sliced(packed, cols: int, bits: int):
+def unpack_sliced(packed, rows: int, cols: int, bits: int):
     packed = _c(packed, np.uint8)
-    rows = packed.shape[0]
-    assert packed.shape[1] == sliced_row_bytes(cols, bits)
+    assert packed.size == sliced_padded_rows(rows) * sliced_row_bytes(cols, bits)
     out = np.empty((rows, cols), dtype=np.int8)
     rc = _load().nqo_unpack_sliced(_p(packed), _i64(rows), _i64(cols), bits, _p(out))
     if rc != 0:

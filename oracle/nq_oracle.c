@@ -194,20 +194,23 @@ void nqo_unpack_word64(const uint64_t *in, int64_t rows, int64_t cols, int bits,
 /* O4b  the "sliced" layout (this library's storage format, not the paper's)  */
 /* ------------------------------------------------------------------------- */
 /*
- * A row of `cols` k-bit two's-complement fields is padded with zero fields to a
- * multiple of 128 and cut into groups of 128 elements.  A group takes 16*k bytes.
- * k is written as a sum of distinct powers of two (8, 4, 2, 1), widest first; each
- * power s is a "slice" that holds s bits of every field, the widest slice holding
- * the most significant bits.  Inside a group the slices follow one another, the
- * slice of width s occupying 16*s bytes.  Inside a slice, element e of the group
- * (0..127) is placed as
+ * A [rows, cols] tensor of k-bit two's-complement fields is padded with zero fields to
+ * multiples of 128 in both directions and cut into blocks of 128 rows x 128 columns.
+ * A block takes 2048*k bytes; blocks follow one another row-block by row-block
+ * (block (rb, g) of a tensor with G = ceil(cols/128) column groups is block number
+ * rb*G + g).  k is written as a sum of distinct powers of two (8, 4, 2, 1), widest
+ * first; each power s is a "slice" that holds s bits of every field, the widest slice
+ * holding the most significant bits.  Inside a block the slices follow one another,
+ * the slice of width s occupying 2048*s bytes: the 128 rows of the block one after the
+ * other, 16*s bytes each.  Inside a row's 16*s bytes, element e of the row's 128
+ * (e = column % 128) is placed as
  *      unit = e / 32        a unit is 32 elements = s little-endian 32-bit words
  *      q    = (e % 32) / 4  which of the unit's eight 4-element quads
  *      lane = e % 4         byte lane inside the word
  *      word = q / (8 / s)   8/s slices share one byte
  *      sub  = q % (8 / s)   sub 0 sits in the TOP bits of the byte
- * i.e. byte (unit*s + word)*4 + lane of the slice, bits [8 - s*sub - s, 8 - s*sub).
- * With s = 8 this is the plain byte order.
+ * i.e. byte (unit*s + word)*4 + lane, bits [8 - s*sub - s, 8 - s*sub).
+ * With s = 8 this is the plain byte order of the block's rows.
  */
 static int slice_widths(int bits, int widths[4])
 {
@@ -217,13 +220,16 @@ static int slice_widths(int bits, int widths[4])
     return n;
 }
 
+/* bytes per row of the padded tensor (a size unit only: a row's bytes are not contiguous) */
 int64_t nqo_sliced_row_bytes(int64_t cols, int bits)
 {
     int64_t groups = (cols + 127) / 128;
     return groups * 16 * bits;
 }
 
-/* where slice `s` of group element `e` lives: byte offset inside the slice, shift inside the byte */
+int64_t nqo_sliced_padded_rows(int64_t rows) { return (rows + 127) / 128 * 128; }
+
+/* where slice `s` keeps the bits of element e of a row: byte offset inside the row's 16*s bytes, shift inside the byte */
 static void slice_place(int s, int e, int64_t *byte_off, int *shift)
 {
     int unit = e / 32, q = (e % 32) / 4, lane = e % 4;
@@ -233,28 +239,32 @@ static void slice_place(int s, int e, int64_t *byte_off, int *shift)
     *shift = 8 - s * sub - s;
 }
 
+/* start of the 16*s bytes that slice number k (preceded by `bits_before` bits of wider slices) keeps for row r, column c */
+static int64_t slice_row_start(int64_t r, int64_t c, int64_t groups, int bits, int bits_before, int s)
+{
+    int64_t block = (r / 128) * groups + c / 128;
+    return block * 2048 * bits + (int64_t)2048 * bits_before + (r % 128) * 16 * s;
+}
+
 int nqo_pack_sliced(const int8_t *v, int64_t rows, int64_t cols, int bits, uint8_t *out)
 {
     if (bits < 1 || bits > 8) return -1;
     int widths[4];
     const int nslices = slice_widths(bits, widths);
-    const int64_t pitch = nqo_sliced_row_bytes(cols, bits);
-    memset(out, 0, (size_t)(rows * pitch));
+    const int64_t groups = (cols + 127) / 128;
+    memset(out, 0, (size_t)(nqo_sliced_padded_rows(rows) * groups * 16 * bits));
     for (int64_t r = 0; r < rows; ++r)
         for (int64_t c = 0; c < cols; ++c) {
             uint32_t field = ((uint32_t)(int32_t)v[r * cols + c]) & ((1u << bits) - 1u);
-            uint8_t *group = out + r * pitch + (c / 128) * 16 * bits;
             int e = (int)(c % 128);
             int consumed = 0;                     /* field bits already placed, from the top */
-            int64_t slice_base = 0;
             for (int k = 0; k < nslices; ++k) {
                 int s = widths[k];
                 uint32_t part = (field >> (bits - consumed - s)) & ((1u << s) - 1u);
                 int64_t off; int sh;
                 slice_place(s, e, &off, &sh);
-                group[slice_base + off] |= (uint8_t)(part << sh);
+                out[slice_row_start(r, c, groups, bits, consumed, s) + off] |= (uint8_t)(part << sh);
                 consumed += s;
-                slice_base += 16 * s;
             }
         }
     return 0;
@@ -265,20 +275,19 @@ int nqo_unpack_sliced(const uint8_t *in, int64_t rows, int64_t cols, int bits, i
     if (bits < 1 || bits > 8) return -1;
     int widths[4];
     const int nslices = slice_widths(bits, widths);
-    const int64_t pitch = nqo_sliced_row_bytes(cols, bits);
+    const int64_t groups = (cols + 127) / 128;
     for (int64_t r = 0; r < rows; ++r)
         for (int64_t c = 0; c < cols; ++c) {
-            const uint8_t *group = in + r * pitch + (c / 128) * 16 * bits;
             int e = (int)(c % 128);
             uint32_t field = 0;
-            int64_t slice_base = 0;
+            int consumed = 0;
             for (int k = 0; k < nslices; ++k) {
                 int s = widths[k];
                 int64_t off; int sh;
                 slice_place(s, e, &off, &sh);
-                uint32_t part = ((uint32_t)group[slice_base + off] >> sh) & ((1u << s) - 1u);
+                uint32_t part = ((uint32_t)in[slice_row_start(r, c, groups, bits, consumed, s) + off] >> sh) & ((1u << s) - 1u);
                 field = (field << s) | part;
-                slice_base += 16 * s;
+                consumed += s;
             }
             int32_t val = (int32_t)field;
             if (val >= (1 << (bits - 1))) val -= (1 << bits);   /* two's complement field */

@@ -126,13 +126,15 @@ def nq_packed_bytes(rows: int, cols: int, bits: int) -> int:
 
 
 def _empty_packed(rows: int, cols: int, bits: int, device) -> torch.Tensor:
-    return torch.empty((rows, max(nq_packed_row_bytes(cols, bits), 0)), dtype=torch.uint8, device=device)
+    """Storage of a packed tensor: nq_packed_bytes(rows, cols, bits) bytes, shaped [rows padded to 128, bytes per row]
+    (a container only: the layout stores 128 x 128 blocks, a row's bytes are not contiguous)."""
+    return torch.empty((-(-rows // 128) * 128, max(nq_packed_row_bytes(cols, bits), 0)), dtype=torch.uint8, device=device)
 
 
 # --------------------------------------------------------------------------- codec
 def nq_decompose(w_int: torch.Tensor, mask: torch.Tensor, n_bits: int, h_bits: int, compensate: bool = True,
                  out_high: Optional[torch.Tensor] = None, out_low: Optional[torch.Tensor] = None):
-    """-> (packed_high, packed_low) uint8 [rows, row_bytes]."""
+    """-> (packed_high, packed_low): uint8 storage of the two sliced tensors."""
     _need(w_int, torch.int8, "w_int", 2)
     _need(mask, torch.uint8, "mask", 2)
     if mask.shape != w_int.shape or _ld(mask) != _ld(w_int):

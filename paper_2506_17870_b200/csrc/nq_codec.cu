@@ -2,7 +2,10 @@
 // the plain pack / unpack test aids, all on the sliced sub-byte layout described in nq.h.
 //
 // Work unit: 32 consecutive elements of one row = eight 32-bit words of int8 on the unpacked side
-// and, per slice of width s, s words on the packed side.  One thread owns one unit at a time and
+// and, per slice of width s, s words on the packed side.  Units are walked block by block (128 rows x 128
+// columns, the packed layout's storage unit), rows fastest: the 32 lanes of a warp hold four units of each of
+// eight consecutive rows, so every packed access of a warp is one contiguous run (512 / 256 / 128 bytes of the
+// 4- / 2- / 1-bit slice) and every int8 access covers eight whole 128-byte lines.  One thread owns one unit at a time and
 // keeps it in registers as eight "top-aligned" words T[q]: byte lane i of T[q] holds the k-bit
 // field of element 4q+i in its TOP k bits.  In that form every slice is a fixed bit range of every
 // byte, so moving between T and the slices is a mask, a shift and an OR per word -- four elements
@@ -87,16 +90,18 @@ struct PackedRaw {
     uint32_t d;      // 1-bit slice
 };
 
-__device__ __forceinline__ void load_packed_raw(const uint8_t* __restrict__ group, int unit, int bits, PackedRaw& r) {
+// `block` is the start of a 128 x 128 block of `bits`-bit fields, `ru` = row-in-block * 4 + unit (0 .. 511): the
+// slice of width s starts 2048 * (bits of the wider slices) bytes into the block and keeps 4 * s bytes per unit.
+__device__ __forceinline__ void load_packed_raw(const uint8_t* __restrict__ block, int ru, int bits, PackedRaw& r) {
     if (bits == 8) {
-        const uint4* p = reinterpret_cast<const uint4*>(group + unit * 32);
+        const uint4* p = reinterpret_cast<const uint4*>(block + ru * 32);
         r.a = __ldg(p); r.b = __ldg(p + 1);
         return;
     }
     int off = 0;
-    if (bits & 4) { r.a = __ldg(reinterpret_cast<const uint4*>(group + unit * 16)); off = 64; }
-    if (bits & 2) { r.c = __ldg(reinterpret_cast<const uint2*>(group + off + unit * 8)); off += 32; }
-    if (bits & 1) { r.d = __ldg(reinterpret_cast<const uint32_t*>(group + off + unit * 4)); }
+    if (bits & 4) { r.a = __ldg(reinterpret_cast<const uint4*>(block + ru * 16)); off = 8192; }
+    if (bits & 2) { r.c = __ldg(reinterpret_cast<const uint2*>(block + off + ru * 8)); off += 4096; }
+    if (bits & 1) { r.d = __ldg(reinterpret_cast<const uint32_t*>(block + off + ru * 4)); }
 }
 
 __device__ __forceinline__ void expand_packed_raw(const PackedRaw& r, int bits, uint32_t (&T)[8]) {
@@ -135,10 +140,10 @@ __device__ __forceinline__ void expand_packed_raw(const PackedRaw& r, int bits, 
     }
 }
 
-__device__ __forceinline__ void store_unit_top(uint8_t* __restrict__ group, int unit, int bits,
+__device__ __forceinline__ void store_unit_top(uint8_t* __restrict__ block, int ru, int bits,
                                                const uint32_t (&T)[8]) {
     if (bits == 8) {
-        uint4* p = reinterpret_cast<uint4*>(group + unit * 32);
+        uint4* p = reinterpret_cast<uint4*>(block + ru * 32);
         p[0] = make_uint4(T[0], T[1], T[2], T[3]);
         p[1] = make_uint4(T[4], T[5], T[6], T[7]);
         return;
@@ -150,8 +155,8 @@ __device__ __forceinline__ void store_unit_top(uint8_t* __restrict__ group, int 
         w.y = (T[2] & 0xf0f0f0f0u) | ((T[3] >> 4) & 0x0f0f0f0fu);
         w.z = (T[4] & 0xf0f0f0f0u) | ((T[5] >> 4) & 0x0f0f0f0fu);
         w.w = (T[6] & 0xf0f0f0f0u) | ((T[7] >> 4) & 0x0f0f0f0fu);
-        *reinterpret_cast<uint4*>(group + unit * 16) = w;
-        off = 64; used = 4;
+        *reinterpret_cast<uint4*>(block + ru * 16) = w;
+        off = 8192; used = 4;
     }
     if (bits & 2) {
         uint2 w = make_uint2(0u, 0u);
@@ -162,8 +167,8 @@ __device__ __forceinline__ void store_unit_top(uint8_t* __restrict__ group, int 
             const uint32_t piece = moved & (0xc0c0c0c0u >> (2 * (q & 3)));
             if (q < 4) w.x |= piece; else w.y |= piece;
         }
-        *reinterpret_cast<uint2*>(group + off + unit * 8) = w;
-        off += 32; used += 2;
+        *reinterpret_cast<uint2*>(block + off + ru * 8) = w;
+        off += 4096; used += 2;
     }
     if (bits & 1) {
         uint32_t w = 0;
@@ -173,7 +178,7 @@ __device__ __forceinline__ void store_unit_top(uint8_t* __restrict__ group, int 
             const uint32_t moved = net >= 0 ? (T[q] << net) : (T[q] >> (-net));
             w |= moved & (H4 >> q);
         }
-        *reinterpret_cast<uint32_t*>(group + off + unit * 4) = w;
+        *reinterpret_cast<uint32_t*>(block + off + ru * 4) = w;
     }
 }
 
@@ -311,65 +316,71 @@ struct TensorView {
 
 enum Op { OP_DECOMPOSE = 0, OP_RECOMPOSE = 1, OP_DROP_LOW = 2, OP_UNPACK = 3, OP_PACK = 4 };
 
+// unit_index counts units block by block: 512 per block (row-in-block * 4 + unit), blocks in storage order.
 template <int OP, class NestT>
 __device__ __forceinline__ void do_unit(const TensorView& t, int64_t unit_index, const NestT& N, int bits) {
-    const int64_t units_per_row = ((t.cols + 127) >> 7) << 2;
-    int64_t row, ur;
-    if (((unit_index | units_per_row) >> 32) == 0) {          // the usual case: 32-bit divide
-        const uint32_t r32 = (uint32_t)unit_index / (uint32_t)units_per_row;
-        row = r32;
-        ur = (uint32_t)unit_index - r32 * (uint32_t)units_per_row;
+    const int64_t groups = (t.cols + 127) >> 7;
+    const int64_t blk = unit_index >> 9;
+    const int ru = (int)(unit_index & 511);
+    int64_t rb, g;
+    if (((blk | groups) >> 32) == 0) {                        // the usual case: 32-bit divide
+        const uint32_t q = (uint32_t)blk / (uint32_t)groups;
+        rb = q;
+        g = (uint32_t)blk - q * (uint32_t)groups;
     } else {
-        row = unit_index / units_per_row;
-        ur = unit_index - row * units_per_row;
+        rb = blk / groups;
+        g = blk - rb * groups;
     }
-    const int64_t group = row * (units_per_row >> 2) + (ur >> 2);
-    const int unit = (int)(ur & 3);
-    const int64_t c0 = ur * 32;
+    const int64_t row = rb * 128 + (ru >> 2);
+    const int64_t c0 = (g * 4 + (ru & 3)) * 32;
+    const bool row_in = row < t.rows;                         // rows of the last block beyond the tensor are padding
+    const bool to_packed = OP == OP_DECOMPOSE || OP == OP_DROP_LOW || OP == OP_PACK;
+    if (!row_in && !to_packed) return;
     const bool vec_ok = ((t.ld & 15) == 0) && ((reinterpret_cast<uintptr_t>(t.w) & 15) == 0) &&
                         (OP != OP_DECOMPOSE || (reinterpret_cast<uintptr_t>(t.mask) & 15) == 0);
     int8_t* wrow = t.w + row * t.ld;
+    const int64_t cols = row_in ? t.cols : 0;                 // a padding row reads nothing: all its fields are zero
     uint32_t A[8], Bv[8];
     PackedRaw p0, p1;
     I8Raw v0, v1;
     if (OP == OP_DECOMPOSE) {
         const int8_t* mrow = reinterpret_cast<const int8_t*>(t.mask) + row * t.ld;
-        load_i8_raw(wrow, c0, t.cols, vec_ok, v0);
-        load_i8_raw(mrow, c0, t.cols, vec_ok, v1);
-        expand_i8_raw(v0, wrow, c0, t.cols, A);
-        expand_i8_raw(v1, mrow, c0, t.cols, Bv);
+        load_i8_raw(wrow, c0, cols, vec_ok, v0);
+        load_i8_raw(mrow, c0, cols, vec_ok, v1);
+        expand_i8_raw(v0, wrow, c0, cols, A);
+        expand_i8_raw(v1, mrow, c0, cols, Bv);
 #pragma unroll
         for (int q = 0; q < 8; ++q) decompose_word(N, A[q], Bv[q], A[q], Bv[q]);
-        store_unit_top(t.hi + group * 16 * N.h, unit, N.h, A);
-        store_unit_top(t.lo + group * 16 * N.lb, unit, N.lb, Bv);
+        store_unit_top(t.hi + blk * 2048 * N.h, ru, N.h, A);
+        store_unit_top(t.lo + blk * 2048 * N.lb, ru, N.lb, Bv);
     } else if (OP == OP_RECOMPOSE) {
-        load_packed_raw(t.hi + group * 16 * N.h, unit, N.h, p0);
-        load_packed_raw(t.lo + group * 16 * N.lb, unit, N.lb, p1);
+        load_packed_raw(t.hi + blk * 2048 * N.h, ru, N.h, p0);
+        load_packed_raw(t.lo + blk * 2048 * N.lb, ru, N.lb, p1);
         expand_packed_raw(p0, N.h, A);
         expand_packed_raw(p1, N.lb, Bv);
 #pragma unroll
         for (int q = 0; q < 8; ++q) A[q] = recompose_word(N, A[q], Bv[q]);
         store_unit_i8(wrow, c0, t.cols, vec_ok, A);
     } else if (OP == OP_DROP_LOW) {
-        load_i8_raw(wrow, c0, t.cols, vec_ok, v0);
-        load_packed_raw(t.lo + group * 16 * N.lb, unit, N.lb, p1);
-        expand_i8_raw(v0, wrow, c0, t.cols, A);
+        load_i8_raw(wrow, c0, cols, vec_ok, v0);
+        load_packed_raw(t.lo + blk * 2048 * N.lb, ru, N.lb, p1);
+        expand_i8_raw(v0, wrow, c0, cols, A);
         expand_packed_raw(p1, N.lb, Bv);
 #pragma unroll
-        for (int q = 0; q < 8; ++q) A[q] = drop_low_word(N, A[q], Bv[q]);
-        store_unit_top(t.hi + group * 16 * N.h, unit, N.h, A);
+        for (int q = 0; q < 8; ++q) A[q] = row_in ? drop_low_word(N, A[q], Bv[q]) : 0u;
+        store_unit_top(t.hi + blk * 2048 * N.h, ru, N.h, A);
     } else if (OP == OP_UNPACK) {
-        load_packed_raw(t.hi + group * 16 * bits, unit, bits, p0);
+        load_packed_raw(t.hi + blk * 2048 * bits, ru, bits, p0);
         expand_packed_raw(p0, bits, A);
 #pragma unroll
         for (int q = 0; q < 8; ++q) A[q] = top_to_values(A[q], bits);
         store_unit_i8(wrow, c0, t.cols, vec_ok, A);
     } else {
-        load_i8_raw(wrow, c0, t.cols, vec_ok, v0);
-        expand_i8_raw(v0, wrow, c0, t.cols, A);
+        load_i8_raw(wrow, c0, cols, vec_ok, v0);
+        expand_i8_raw(v0, wrow, c0, cols, A);
 #pragma unroll
         for (int q = 0; q < 8; ++q) A[q] = values_to_top(A[q], bits);
-        store_unit_top(t.hi + group * 16 * bits, unit, bits, A);
+        store_unit_top(t.hi + blk * 2048 * bits, ru, bits, A);
     }
 }
 
@@ -392,15 +403,10 @@ struct BatchEntry {
 };
 static_assert(sizeof(BatchEntry) == 64, "table entry is 64 bytes");
 
-// A model is cut into work items of at most kItemUnits units, none of which straddles two tensors; block b of
-// the batched launch takes item b, so no thread ever searches the tensor table.
-#ifndef NQ_ITEM_UNITS
-#define NQ_ITEM_UNITS 512
-#endif
-#ifndef NQ_BATCH_BLOCKS_PER_SM
-#define NQ_BATCH_BLOCKS_PER_SM 4
-#endif
-constexpr int kItemUnits = NQ_ITEM_UNITS;
+// A model is cut into work items of one 128 x 128 block (512 units) each, none of which straddles two tensors;
+// block b of the batched launch takes items b, b + grid, ..., so no thread ever searches the tensor table.
+constexpr int kItemUnits = 512;
+constexpr int kBatchBlocksPerSM = 4;
 struct BatchItem {
     int32_t entry;          // which tensor
     int32_t units;          // how many units of it (<= kItemUnits)
@@ -431,16 +437,19 @@ __global__ void __launch_bounds__(256) word64_to_sliced_kernel(const uint64_t* _
                                                                int64_t cols, uint8_t* __restrict__ packed) {
     constexpr int PER = 64 / BITS;
     constexpr uint32_t MASK = (1u << BITS) - 1u;
-    const int64_t units_per_row = ((cols + 127) >> 7) << 2;
+    const int64_t groups = (cols + 127) >> 7;
+    const int64_t units_per_row = groups << 2;
     const int64_t row_words = (cols + PER - 1) / PER;
-    const int64_t total = rows * units_per_row;
+    const int64_t rows_pad = (rows + 127) / 128 * 128;          // the padding rows of the last block are written as zeros
+    const int64_t total = rows_pad * units_per_row;
     for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < total; u += (int64_t)gridDim.x * blockDim.x) {
         const int64_t row = u / units_per_row, ur = u - row * units_per_row;
         const int64_t c0 = ur * 32;
         const uint64_t* wrow = words + row * row_words;
+        const int64_t cols_here = row < rows ? cols : 0;
         int64_t wi = c0 / PER;
         int fi = (int)(c0 - wi * PER);
-        uint64_t w = (c0 < cols) ? __ldg(wrow + wi) >> (fi * BITS) : 0ull;
+        uint64_t w = (c0 < cols_here) ? __ldg(wrow + wi) >> (fi * BITS) : 0ull;
         uint32_t T[8];
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
@@ -448,18 +457,18 @@ __global__ void __launch_bounds__(256) word64_to_sliced_kernel(const uint64_t* _
 #pragma unroll
             for (int lane = 0; lane < 4; ++lane) {
                 const int j = q * 4 + lane;
-                const uint32_t f = (c0 + j < cols) ? ((uint32_t)w & MASK) : 0u;
+                const uint32_t f = (c0 + j < cols_here) ? ((uint32_t)w & MASK) : 0u;
                 t |= f << (8 * lane + 8 - BITS);
                 w >>= BITS;
                 if (++fi == PER) {
                     fi = 0;
                     ++wi;
-                    w = (c0 + j + 1 < cols) ? __ldg(wrow + wi) : 0ull;
+                    w = (c0 + j + 1 < cols_here) ? __ldg(wrow + wi) : 0ull;
                 }
             }
             T[q] = t;
         }
-        store_unit_top(packed + (row * (units_per_row >> 2) + (ur >> 2)) * 16 * BITS, (int)(ur & 3), BITS, T);
+        store_unit_top(packed + ((row >> 7) * groups + (ur >> 2)) * 2048 * BITS, (int)((row & 127) * 4 + (ur & 3)), BITS, T);
     }
 }
 
@@ -483,7 +492,7 @@ void launch_batch(const BatchEntry* table, int count, int64_t items, int n, int 
     // as many blocks as are resident at once (four per SM); a block walks the items b, b + grid, ...: with small
     // items the last round is a small part of the whole, where one block per item of 1024 units left the
     // ResNet-101-shaped model with 2.3 rounds of blocks
-    const int64_t resident = (int64_t)nq::sm_count() * NQ_BATCH_BLOCKS_PER_SM;
+    const int64_t resident = (int64_t)nq::sm_count() * kBatchBlocksPerSM;
     const unsigned grid = (unsigned)(items < resident ? items : resident);
     codec_batched_kernel<OP, NestT><<<grid, 256, 0, s>>>(table, list, (int)items, n, h, comp);
 }
@@ -521,7 +530,7 @@ void dispatch_nest(bool batched, const TensorView& t, const BatchEntry* table, i
 template <int OP>
 int run_single(TensorView t, int n, int h, int comp, int bits, void* stream) {
     if (t.rows == 0 || t.cols == 0) return NQ_OK;
-    int64_t total = t.rows * ((t.cols + 127) / 128) * 4;
+    int64_t total = ((t.rows + 127) / 128) * ((t.cols + 127) / 128) * 512;       // whole blocks, 512 units each
     if (OP == OP_UNPACK || OP == OP_PACK) launch_one<OP, Nest>(t, total, n, h, comp, bits, (cudaStream_t)stream);
     else dispatch_nest<OP>(false, t, nullptr, 0, total, n, h, comp, (cudaStream_t)stream);
     return cudaGetLastError() == cudaSuccess ? NQ_OK : NQ_ERR_CUDA;
@@ -531,7 +540,7 @@ int run_single(TensorView t, int n, int h, int comp, int bits, void* stream) {
 
 namespace nq {
 int word64_to_sliced_launch(const uint64_t* words, int bits, int64_t rows, int64_t cols, uint8_t* packed, cudaStream_t s) {
-    const int64_t units = rows * (((cols + 127) >> 7) << 2);
+    const int64_t units = ((rows + 127) / 128 * 128) * (((cols + 127) >> 7) << 2);
     const int blocks = launch_blocks(units);
     switch (bits) {
         case 1: word64_to_sliced_kernel<1><<<blocks, 256, 0, s>>>(words, rows, cols, packed); break;
@@ -562,7 +571,7 @@ int64_t nq_packed_row_bytes(int64_t cols, int bits) {
 int64_t nq_packed_bytes(int64_t rows, int64_t cols, int bits) {
     if (rows < 0) return -1;
     int64_t r = nq_packed_row_bytes(cols, bits);
-    return r < 0 ? -1 : r * rows;
+    return r < 0 ? -1 : r * ((rows + 127) / 128 * 128);
 }
 
 int nq_decompose(const int8_t* w_int, const uint8_t* mask, int64_t rows, int64_t cols, int64_t ld_w,
@@ -619,8 +628,7 @@ int nq_pack(const int8_t* values, int64_t ld, int bits, int64_t rows, int64_t co
 }
 
 static int64_t items_of(const nq_tensor_desc& d) {
-    const int64_t units = d.rows * ((d.cols + 127) / 128) * 4;
-    return (units + kItemUnits - 1) / kItemUnits;
+    return ((d.rows + 127) / 128) * ((d.cols + 127) / 128);              // one item per 128 x 128 block
 }
 
 int64_t nq_batch_table_bytes(const nq_tensor_desc* descs, int count) {
@@ -656,7 +664,7 @@ int nq_batch_plan(const nq_tensor_desc* descs, int count, void* table, int64_t t
         e.rows = d.rows; e.cols = d.cols; e.ld = d.ld;
         e.hi = (uint8_t*)d.packed_high; e.lo = (uint8_t*)d.packed_low; e.w = d.w_int;
         e.first_unit = units_before; e.pad_ = 0;
-        const int64_t units = d.rows * ((d.cols + 127) / 128) * 4;
+        const int64_t units = items_of(d) * kItemUnits;
         units_before += units;
         for (int64_t u = 0; u < units; u += kItemUnits) {
             BatchItem& it = items[n_items++];

@@ -77,14 +77,17 @@ struct ContractionArgs {
     int acc_shift;       // 8-h in part-bit mode, 0 otherwise
     int h_bits;          // part-bit: width of the packed field
     int packed_stages;   // part-bit: depth of the packed-tile ring (1..kMaxPackedStages)
-    const uint8_t* packed_b;   // part-bit: the packed matrix itself and its row pitch in bytes
-    long long packed_pitch;
-    int ring_bits;       // pair kernel: bits per field in a packed-ring tile (h_bits in part-bit mode; in nested
-                         // full-bit mode the wider of the two fields, plus one when ring2 is set; packed_b is then
-                         // the tensor of the narrower field)
-    int ring_x_bytes;    // ... bytes per 128-field group of the tensor behind tmB
-    int ring2;           // nested mode, 3-bit narrow field: its 1-bit slice is loaded into the ring tile as well,
-                         // through the map passed in the tmAcc slot (accumulators then take ordinary stores)
+    // Packed operands (part-bit, nested): tensors in the sliced layout, blocks of 128 rows x 128 fields, 2048 * bits
+    // contiguous bytes each, block (rb, g) at ((rb * packed_groups + g) * 2048 * bits).
+    const uint8_t* packed_b;   // the tensor the unpack warps read straight from global memory (part-bit: packed_high; nested:
+                               // the narrower of the two fields)
+    const uint8_t* ring_b;     // the tensor that comes through the shared-memory ring (part-bit: packed_high; nested: the wider field)
+    int packed_groups;         // column groups G = ceil(K / 128) of both
+    int packed_blocks;         // row blocks ceil(N / 128) that exist; a tile may reach one block further, which is not read
+    int ring_bits;       // bits per field of a ring slot (h_bits in part-bit mode; in nested full-bit mode the wider of the two
+                         // fields, plus one when ring2 is set)
+    int ring_field_bits; // ... of the tensor behind ring_b
+    int ring2;           // nested mode, 3-bit narrow field: its 1-bit slice is copied into the ring slot as well
     int32_t* acc_out;
     long long ld_acc;
     void* y;
@@ -149,12 +152,14 @@ struct PackedUnit {
     uint2 c;       // 2-bit slice
     uint32_t d;    // 1-bit slice
 };
-template <int H>
-__device__ __forceinline__ void load_packed_unit(const uint8_t* group, int unit, PackedUnit& r) {
+// Out of a ring slot holding ROWS rows of a block slice by slice ([ROWS][64 B] of the 4-bit slice, [ROWS][32 B] of the
+// 2-bit slice, [ROWS][16 B] of the 1-bit slice): unit ru = row * 4 + unit.  Consecutive lanes read consecutive pieces.
+template <int H, int ROWS>
+__device__ __forceinline__ void load_packed_unit(const uint8_t* slot, int ru, PackedUnit& r) {
     int off = 0;
-    if (H & 4) { r.a = *reinterpret_cast<const uint4*>(group + unit * 16); off = 64; }
-    if (H & 2) { r.c = *reinterpret_cast<const uint2*>(group + off + unit * 8); off += 32; }
-    if (H & 1) { r.d = *reinterpret_cast<const uint32_t*>(group + off + unit * 4); }
+    if (H & 4) { r.a = *reinterpret_cast<const uint4*>(slot + ru * 16); off = ROWS * 64; }
+    if (H & 2) { r.c = *reinterpret_cast<const uint2*>(slot + off + ru * 8); off += ROWS * 32; }
+    if (H & 1) { r.d = *reinterpret_cast<const uint32_t*>(slot + off + ru * 4); }
 }
 // ... and its expansion to 32 bytes with the field in the TOP H bits of each byte.  All shifts and masks are
 // immediates: the 4-bit slice costs one AND (or shift + AND) per word, every narrower slice one shift and one
@@ -264,27 +269,29 @@ __device__ __forceinline__ void store_expanded_unit(uint8_t* __restrict__ dst, i
     }
 }
 
-// The same unit fetched straight from the packed matrix in global memory (group = start of the row's
-// 128-field group); a row past the end of the matrix reads as zeros.
+// The same unit fetched straight from a block of the packed tensor in global memory (ru = row-in-block * 4 + unit):
+// the 32 lanes of a warp read 512 / 256 / 128 contiguous bytes.  A row past the end of the matrix reads as zeros.
 template <int H>
-__device__ __forceinline__ void fetch_packed_unit(const uint8_t* group, int unit, bool in_range, PackedUnit& r) {
+__device__ __forceinline__ void fetch_packed_unit(const uint8_t* block, int ru, bool in_range, PackedUnit& r) {
     r.a = make_uint4(0u, 0u, 0u, 0u); r.c = make_uint2(0u, 0u); r.d = 0u;
     if (!in_range) return;
     int off = 0;
-    if (H & 4) { r.a = sm100::ldg_stream_v4(group + unit * 16); off = 64; }
-    if (H & 2) { r.c = sm100::ldg_stream_v2(group + off + unit * 8); off += 32; }
-    if (H & 1) { r.d = sm100::ldg_stream_u32(group + off + unit * 4); }
+    if (H & 4) { r.a = sm100::ldg_stream_v4(block + ru * 16); off = 8192; }
+    if (H & 2) { r.c = sm100::ldg_stream_v2(block + off + ru * 8); off += 4096; }
+    if (H & 1) { r.d = sm100::ldg_stream_u32(block + off + ru * 4); }
 }
 
 constexpr int kUnpackWarps = 8;
 constexpr int kUnpackThreads = kUnpackWarps * 32;
 
-// Expand one packed B tile (ROWS rows x 128 fields) into the swizzled int8 tile the MMA reads, with THREADS
-// threads (tid = 0 .. THREADS-1); four consecutive threads share a row.
+// Expand one packed B tile (ROWS rows x 128 fields, in a ring slot) into the swizzled int8 tile the MMA reads, with
+// THREADS threads (tid = 0 .. THREADS-1); four consecutive threads share a row.  A slot holds SLOT_ROWS rows slice by
+// slice; tiles of 256 rows are two such runs (two blocks of the packed tensor), one after the other.
 template <int ROWS, int MODE, int H, int THREADS>
 __device__ __forceinline__ void unpack_tile(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, int tid) {
     constexpr int TASKS = ROWS * 4 / THREADS;              // units per thread
     constexpr int CHUNK = TASKS < 4 ? TASKS : 4;           // units whose loads are issued together
+    constexpr int SLOT_ROWS = ROWS < 128 ? ROWS : 128;
     static_assert(TASKS >= 1 && TASKS % CHUNK == 0, "tile does not divide over the threads");
 #pragma unroll
     for (int base = 0; base < TASKS; base += CHUNK) {
@@ -292,7 +299,7 @@ __device__ __forceinline__ void unpack_tile(const uint8_t* __restrict__ src, uin
 #pragma unroll
         for (int i = 0; i < CHUNK; ++i) {
             const int task = (base + i) * THREADS + tid;
-            load_packed_unit<H>(src + (task >> 2) * 16 * H, task & 3, raw[i]);
+            load_packed_unit<H, SLOT_ROWS>(src + (task >> 9) * (2048 * H), task & 511, raw[i]);
         }
 #pragma unroll
         for (int i = 0; i < CHUNK; ++i) {
@@ -301,6 +308,34 @@ __device__ __forceinline__ void unpack_tile(const uint8_t* __restrict__ src, uin
             uint32_t T[8];
             expand_packed_unit<H>(raw[i], T);
             store_expanded_unit<ROWS, MODE>(dst, row, unit, T);
+        }
+    }
+}
+
+// The packed-tile producer's copies of one ring slot of a ROWS-row tile whose first row is row0 (a multiple of ROWS):
+// whole blocks for tiles of 128 and 256 rows, the tile's 64 rows of every slice for tiles of 64 rows.  A block beyond
+// the tensor's last is not copied (its rows are beyond N: their products are never stored).  Announces the bytes first.
+template <int ROWS>
+__device__ __forceinline__ void load_ring_slot(const ContractionArgs& p, uint32_t slot, int row0, int group, uint32_t bar) {
+    const int fb = p.ring_field_bits;
+    if (ROWS >= 128) {
+        const int rb0 = row0 >> 7;
+        int n = 0;
+        for (int j = 0; j < ROWS / 128; ++j) n += (rb0 + j < p.packed_blocks) ? 1 : 0;
+        sm100::mbar_arrive_expect_tx(bar, (uint32_t)(n * 2048 * fb));
+        for (int j = 0; j < ROWS / 128; ++j)
+            if (rb0 + j < p.packed_blocks)
+                sm100::bulk_load(slot + j * 2048 * fb, p.ring_b + ((long long)(rb0 + j) * p.packed_groups + group) * (2048 * fb),
+                                 2048 * fb, bar);
+    } else {
+        const uint8_t* block = p.ring_b + ((long long)(row0 >> 7) * p.packed_groups + group) * (2048 * fb);
+        const int r0 = row0 & 127;
+        sm100::mbar_arrive_expect_tx(bar, (uint32_t)(ROWS * 16 * fb));
+        int done = 0;                                   // bits of the wider slices already placed
+        for (int w = 4; w >= 1; w >>= 1) {
+            if (!(fb & w)) continue;
+            sm100::bulk_load(slot + ROWS * 16 * done, block + 2048 * done + r0 * 16 * w, ROWS * 16 * w, bar);
+            done += w;
         }
     }
 }
@@ -882,9 +917,7 @@ contraction_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++pit) {
                     const uint32_t ps = pit % p.packed_stages, puse = pit / p.packed_stages;
                     if (!(ok = mbar_wait(smem_u32(&pempty[ps]), (puse & 1) ^ 1, abort_flag, p.status, 0x11u))) break;
-                    const uint32_t pb = smem_u32(&pfull[ps]);
-                    mbar_arrive_expect_tx(pb, packed_bytes);
-                    tma_load_2d(smem_u32(sP + ps * packed_bytes), &tmB, kb * 16 * p.h_bits, nt * BN, pb);
+                    load_ring_slot<BN>(p, smem_u32(sP + ps * packed_bytes), nt * BN, kb, smem_u32(&pfull[ps]));
                 }
             }
             if (!ok) {

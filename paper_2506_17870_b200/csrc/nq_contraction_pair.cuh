@@ -90,20 +90,21 @@ __device__ __forceinline__ void advance_cursor(StageCursor& c, int steps, int k_
     while (c.kb >= k_blocks && c.tile < num_tiles) { c.kb -= k_blocks; c.tile += num_pairs; }
 }
 
-// The packed fields of one stage (this CTA's 128 rows of B x one 128-field group) into registers.
-// GROUP_BITS > H: only the leading H bits' worth of slices of a tensor of GROUP_BITS-bit fields (they start the group).
+// The packed fields of one stage (this CTA's 128 rows of B x one 128-field group: one block of the packed tensor,
+// contiguous in memory) into registers.  GROUP_BITS > H: only the leading H bits' worth of slices of a tensor of
+// GROUP_BITS-bit fields (they start the block).
 template <int H, int GROUP_BITS = H>
 __device__ __forceinline__ void fetch_stage(const ContractionArgs& p, const PairUnpackCtx& cx, const StageCursor& c,
                                             PackedUnit (&raw)[kPairUnitsPerThread]) {
     int mt2, nt;
     tile_coords(c.tile, p, mt2, nt);
-    const int brow = nt * kPairBN + (int)cx.rank * (kPairBN / 2);
-    const uint8_t* base = p.packed_b + (long long)c.kb * (16 * GROUP_BITS);
+    const int rb = nt * 2 + (int)cx.rank;                       // this CTA's row block of B
+    const int brow = rb * (kPairBN / 2);
+    const uint8_t* block = p.packed_b + ((long long)rb * p.packed_groups + c.kb) * (2048 * GROUP_BITS);
 #pragma unroll
     for (int i = 0; i < kPairUnitsPerThread; ++i) {
         const int task = i * kUnpackGroupThreads + cx.utid;
-        const int row = brow + (task >> 2);
-        fetch_packed_unit<H>(base + (long long)row * p.packed_pitch, task & 3, row < p.N, raw[i]);
+        fetch_packed_unit<H>(block, task, brow + (task >> 2) < p.N, raw[i]);
     }
 }
 
@@ -179,10 +180,10 @@ __device__ __forceinline__ void pair_unpack_nested(const ContractionArgs& p, con
         for (int i = 0; i < kPairUnitsPerThread; ++i) {
             const int task = i * kUnpackGroupThreads + cx.utid;
             PackedUnit ring;
-            load_packed_unit<RING_BITS>(src + (task >> 2) * 16 * RING_BITS, task & 3, ring);
+            load_packed_unit<RING_BITS, HALF>(src, task, ring);
             PackedUnit narrow = raw[i];
             if (BIT_IN_RING)
-                narrow.d = *reinterpret_cast<const uint32_t*>(src + HALF * 16 * RING_BITS + (task >> 2) * 16 + (task & 3) * 4);
+                narrow.d = *reinterpret_cast<const uint32_t*>(src + HALF * 16 * RING_BITS + task * 4);
             uint32_t T[8], L[8];
             expand_packed_unit<H>(HIGH_IN_RING ? ring : narrow, T);
             expand_packed_unit_at<L1, NB - L1>(HIGH_IN_RING ? narrow : ring, L);
@@ -265,7 +266,7 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
         prefetch_tensormap(&tmA);
         prefetch_tensormap(&tmB);
         if (p.y_tma) prefetch_tensormap(&tmY);
-        if (p.acc_tma || (NEST != 0 && p.ring2)) prefetch_tensormap(&tmAcc);
+        if (p.acc_tma) prefetch_tensormap(&tmAcc);
     }
     if (warp == 1) {
         tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS);
@@ -338,10 +339,15 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
                     const uint32_t ps = pit % p.packed_stages, puse = pit / p.packed_stages;
                     if (!(ok = mbar_wait(smem_u32(&pempty[ps]), (puse & 1) ^ 1, abort_flag, p.status, 0x111u))) break;
                     const uint32_t pb = smem_u32(&pfull[ps]);
-                    mbar_arrive_expect_tx(pb, packed_bytes);
-                    tma_load_2d(smem_u32(sP + ps * packed_bytes), &tmB, kb * p.ring_x_bytes, brow, pb);
-                    if (NEST != 0 && p.ring2)     // the 1-bit slice of a 3-bit narrow field (tmAcc is its map here)
-                        tma_load_2d(smem_u32(sP + ps * packed_bytes + HALF * p.ring_x_bytes), &tmAcc, kb * 48 + 32, brow, pb);
+                    const int rb = brow >> 7;
+                    const bool extra = NEST != 0 && p.ring2 && rb < p.packed_blocks;
+                    // the 1-bit slice of a 3-bit narrow field rides behind the wide field's block: 128 rows x 16 bytes, the
+                    // last 2048 bytes of the narrow tensor's block
+                    if (extra) mbar_expect_tx(pb, 2048);
+                    load_ring_slot<HALF>(p, smem_u32(sP + ps * packed_bytes), brow, kb, pb);
+                    if (extra)
+                        bulk_load(smem_u32(sP + ps * packed_bytes + 2048 * p.ring_field_bits),
+                                  p.packed_b + ((long long)rb * p.packed_groups + kb) * (2048 * 3) + 4096, 2048, pb);
                 }
             }
             if (!ok) {
@@ -405,7 +411,10 @@ contraction_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_co
             case 1: pair_unpack_direct<MODE, 1>(p, cx); break;
             case 2: pair_unpack_direct<MODE, 2>(p, cx); break;
             case 3: pair_unpack_direct<MODE, 3>(p, cx); break;
-            default: pair_unpack_direct<MODE, 4>(p, cx); break;
+            case 4: pair_unpack_direct<MODE, 4>(p, cx); break;
+            case 5: pair_unpack_direct<MODE, 5>(p, cx); break;
+            case 6: pair_unpack_direct<MODE, 6>(p, cx); break;
+            default: pair_unpack_direct<MODE, 7>(p, cx); break;
         }
     } else if (PART && NEST != 0 && warp < kPackedProducerWarp) {
         // ------------------------------------------------------------------ unpackers joining both parts (Eq. 5)

@@ -251,9 +251,8 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
         // as deep a ring of packed tiles as shared memory allows: it is what hides the load latency of B
         // (pair kernel: a multiple of its unpack group count, see nq_contraction_pair.cuh)
         a.packed_stages = 0;
-        // direct reads for h = 1, 2, 4 (one load per 32 fields); h = 3 needs two and runs faster through the ring
-        // (8192^3, same box: 3.14 against 2.71 POP/s)
-        direct = !nest && pair && h_bits <= 4 && h_bits != 3 && direct_fetch_enabled();
+        // pair kernel, part-bit: every width is read straight from the packed tensor's blocks (contiguous, coalesced)
+        direct = !nest && pair && direct_fetch_enabled();
         const bool high_in_ring = !nest || h_bits > l + 1;
         const int ring_bits = high_in_ring ? h_bits : l + 1;
         const int direct_bits = nest ? (high_in_ring ? l + 1 : h_bits) : h_bits;
@@ -261,15 +260,8 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
         const void* direct_mat = nest ? (high_in_ring ? Blow : Bmat) : Bmat;
         const bool ring2 = nest && direct_bits == 3;
         a.ring2 = ring2 ? 1 : 0;
+        a.ring_field_bits = ring_bits;
         a.ring_bits = ring_bits + (ring2 ? 1 : 0);
-        a.ring_x_bytes = 16 * ring_bits;
-        if (ring2) {
-            // the narrow tensor's 1-bit slice: 16 bytes per row and group, at byte 32 of every 48-byte group
-            const uint64_t nrow = (uint64_t)((K + 127) / 128) * 48;
-            int st2 = encode_tensor_map_2d(&om.acc, direct_mat, nrow, (uint64_t)N, nrow, 16, b_box_rows, 0);
-            if (st2 != NQ_OK) return st2;
-            a.acc_tma = 0;
-        }
         const int step = pair ? kUnpackGroups : 1;
         for (int d = direct ? 0 : kMaxPackedStages; d >= step; d -= step)
             if ((pair ? pair_smem_bytes(true, a.ring_bits, d) : contraction_smem_bytes(bn, true, h_bits, d)) <= kSmemLimit) {
@@ -277,11 +269,11 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
                 break;
             }
         if (a.packed_stages == 0 && !direct) return NQ_ERR_UNSUPPORTED;
-        const uint64_t row_bytes = (uint64_t)((K + 127) / 128) * 16 * ring_bits;
         a.packed_b = static_cast<const uint8_t*>(direct_mat);     // read directly by the unpack warps (DIRECT, nested)
-        a.packed_pitch = (long long)((K + 127) / 128) * 16 * direct_bits;
-        int st = encode_tensor_map_2d(&tmB, ring_mat, row_bytes, (uint64_t)N, row_bytes, 16 * ring_bits, b_box_rows, 0);
-        if (st != NQ_OK) return st;
+        a.ring_b = static_cast<const uint8_t*>(ring_mat);         // copied block by block into the ring of packed tiles
+        a.packed_groups = (int)((K + 127) / 128);
+        a.packed_blocks = (int)((N + 127) / 128);
+        tmB = tmA;                                                // packed operands need no tensor map: blocks are contiguous
     } else {
         a.pow2_l = 1.0f; a.unshift = 1.0f; a.acc_shift = 0; a.h_bits = 0;
         int st = (mode == kModeConv64)

@@ -16,8 +16,8 @@
 
 namespace {
 
-// Where slice `s` (a power of two) keeps the bits of group element e: byte offset inside the slice and shift
-// inside that byte (the first of the 8/s fields that share a byte sits in its top bits).
+// Where slice `s` (a power of two) keeps the bits of element e of a row's 128: byte offset inside the row's 16 * s
+// bytes of that slice and shift inside that byte (the first of the 8/s fields that share a byte sits in its top bits).
 __device__ __forceinline__ void slice_place(int s, int e, int& byte_off, int& shift) {
     const int unit = e >> 5, q = (e & 31) >> 2, lane = e & 3;
     const int per_byte = 8 / s;
@@ -40,8 +40,9 @@ __global__ void __launch_bounds__(256) sliced_to_word64_kernel(const uint8_t* __
         for (int j = 0; j < PER; ++j) {
             const int64_t c = wd * PER + j;
             if (c >= cols) break;
-            const uint8_t* group = packed + (row * groups_per_row + (c >> 7)) * 16 * BITS;
-            const int e = (int)(c & 127);
+            // block (row / 128, column group), 2048 * BITS bytes; in it the slices, each 128 rows of 16 * s bytes
+            const uint8_t* block = packed + ((row >> 7) * groups_per_row + (c >> 7)) * 2048 * BITS;
+            const int e = (int)(c & 127), r = (int)(row & 127);
             uint32_t field = 0;
             int slice_base = 0;
 #pragma unroll
@@ -49,8 +50,8 @@ __global__ void __launch_bounds__(256) sliced_to_word64_kernel(const uint8_t* __
                 if (!(BITS & s)) continue;
                 int off, sh;
                 slice_place(s, e, off, sh);
-                field = (field << s) | ((uint32_t)(group[slice_base + off] >> sh) & ((1u << s) - 1u));
-                slice_base += 16 * s;
+                field = (field << s) | ((uint32_t)(block[slice_base + r * 16 * s + off] >> sh) & ((1u << s) - 1u));
+                slice_base += 2048 * s;
             }
             out |= (uint64_t)field << (j * BITS);
         }

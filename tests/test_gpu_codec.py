@@ -84,16 +84,16 @@ def test_recompose_and_drop_low_on_arbitrary_bytes(n, h, comp):
     rng = wl.rng_for(93, n * 10 + h)
     lb = n - h + comp
     rows, cols = 37, 384
-    hi = rng.integers(0, 256, size=(rows, oracle.sliced_row_bytes(cols, h)), dtype=np.uint8)
-    lo = rng.integers(0, 256, size=(rows, oracle.sliced_row_bytes(cols, lb)), dtype=np.uint8)
-    wh, wl_ = oracle.unpack_sliced(hi, cols, h), oracle.unpack_sliced(lo, cols, lb)
+    pad = oracle.sliced_padded_rows(rows)
+    hi = rng.integers(0, 256, size=(pad, oracle.sliced_row_bytes(cols, h)), dtype=np.uint8)
+    lo = rng.integers(0, 256, size=(pad, oracle.sliced_row_bytes(cols, lb)), dtype=np.uint8)
+    wh, wl_ = oracle.unpack_sliced(hi, rows, cols, h), oracle.unpack_sliced(lo, rows, cols, lb)
     got = host(nq.nq_recompose(dev(hi), dev(lo), rows, cols, n, h, bool(comp)))
     assert np.array_equal(got, oracle.recompose(wh, wl_, n, h))
     w = rand_weights(rng, (rows, cols), n)
     got_hi = host(nq.nq_drop_low(dev(w), dev(lo), n, h, bool(comp)))
     want = oracle.drop_low(w, wl_, n, h)
-    assert np.array_equal(oracle.unpack_sliced(got_hi, cols, h),
-                          oracle.unpack_sliced(oracle.pack_sliced(want, h), cols, h))
+    assert np.array_equal(got_hi, oracle.pack_sliced(want, h))     # padding rows and columns included: zero fields
 
 
 def test_paper_invariants_on_the_gpu_at_config1_size():
@@ -165,7 +165,15 @@ def test_large_tensor_sampled_against_the_oracle():
     hi, lo = nq.nq_decompose(dev(w), dev(mask), 8, 5, True)
     rec = nq.nq_recompose(hi, lo, rows, cols, 8, 5, True)
     assert torch.equal(rec, dev(w))
+    # the packed bytes of three whole row blocks (a row block's 128 x 128 blocks are contiguous in storage) ...
+    for rb in (0, 17, rows // 128 - 1):
+        band = slice(rb * 128, rb * 128 + 128)
+        wh, wl_ = oracle.decompose(w[band], mask[band], 8, 5, True)
+        assert np.array_equal(host(hi[band]), oracle.pack_sliced(wh, 5))
+        assert np.array_equal(host(lo[band]), oracle.pack_sliced(wl_, 4))
+    # ... and the field values of sampled rows anywhere
     sample = np.unique(np.concatenate([[0, 1, 127, 128, rows - 1], rng.integers(0, rows, 40)]))
     wh, wl_ = oracle.decompose(w[sample], mask[sample], 8, 5, True)
-    assert np.array_equal(host(hi[torch.from_numpy(sample).cuda()]), oracle.pack_sliced(wh, 5))
-    assert np.array_equal(host(lo[torch.from_numpy(sample).cuda()]), oracle.pack_sliced(wl_, 4))
+    idx = torch.from_numpy(sample).cuda()
+    assert np.array_equal(host(nq.nq_unpack(hi, 5, rows, cols)[idx]), wh)
+    assert np.array_equal(host(nq.nq_unpack(lo, 4, rows, cols)[idx]), wl_)

@@ -37,7 +37,8 @@ def test_host_side_size_functions(library):
     assert nq.nq_packed_row_bytes(147, 6) == 192
     assert nq.nq_packed_row_bytes(0, 6) == 0
     assert nq.nq_packed_row_bytes(10, 9) == -1
-    assert nq.nq_packed_bytes(64, 576, 3) == 64 * 5 * 48
+    assert nq.nq_packed_bytes(64, 576, 3) == 128 * 5 * 48          # rows padded to a whole 128-row block
+    assert nq.nq_packed_bytes(129, 128, 8) == 256 * 128
     assert nq.status_str(0) == "ok" and "alignment" in nq.status_str(3)
 
 
