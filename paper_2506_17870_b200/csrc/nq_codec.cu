@@ -316,46 +316,30 @@ struct TensorView {
 
 enum Op { OP_DECOMPOSE = 0, OP_RECOMPOSE = 1, OP_DROP_LOW = 2, OP_UNPACK = 3, OP_PACK = 4 };
 
-// unit_index counts units block by block: 512 per block (row-in-block * 4 + unit), blocks in storage order.
+// One unit: `hi` / `lo` point at the unit's block of the respective packed tensor, ru = row-in-block * 4 + unit,
+// wrow at the int8 row, c0 is the unit's first column.  A row beyond the tensor (padding of the last row block) is
+// written as zero fields by the kernels that produce packed tensors and skipped by the others.
 template <int OP, class NestT>
-__device__ __forceinline__ void do_unit(const TensorView& t, int64_t unit_index, const NestT& N, int bits) {
-    const int64_t groups = (t.cols + 127) >> 7;
-    const int64_t blk = unit_index >> 9;
-    const int ru = (int)(unit_index & 511);
-    int64_t rb, g;
-    if (((blk | groups) >> 32) == 0) {                        // the usual case: 32-bit divide
-        const uint32_t q = (uint32_t)blk / (uint32_t)groups;
-        rb = q;
-        g = (uint32_t)blk - q * (uint32_t)groups;
-    } else {
-        rb = blk / groups;
-        g = blk - rb * groups;
-    }
-    const int64_t row = rb * 128 + (ru >> 2);
-    const int64_t c0 = (g * 4 + (ru & 3)) * 32;
-    const bool row_in = row < t.rows;                         // rows of the last block beyond the tensor are padding
+__device__ __forceinline__ void unit_body(const TensorView& t, const NestT& N, int bits, uint8_t* hi, uint8_t* lo, int ru,
+                                          int8_t* wrow, const int8_t* mrow, uint32_t c0, bool row_in, bool vec_ok) {
     const bool to_packed = OP == OP_DECOMPOSE || OP == OP_DROP_LOW || OP == OP_PACK;
     if (!row_in && !to_packed) return;
-    const bool vec_ok = ((t.ld & 15) == 0) && ((reinterpret_cast<uintptr_t>(t.w) & 15) == 0) &&
-                        (OP != OP_DECOMPOSE || (reinterpret_cast<uintptr_t>(t.mask) & 15) == 0);
-    int8_t* wrow = t.w + row * t.ld;
     const int64_t cols = row_in ? t.cols : 0;                 // a padding row reads nothing: all its fields are zero
     uint32_t A[8], Bv[8];
     PackedRaw p0, p1;
     I8Raw v0, v1;
     if (OP == OP_DECOMPOSE) {
-        const int8_t* mrow = reinterpret_cast<const int8_t*>(t.mask) + row * t.ld;
         load_i8_raw(wrow, c0, cols, vec_ok, v0);
         load_i8_raw(mrow, c0, cols, vec_ok, v1);
         expand_i8_raw(v0, wrow, c0, cols, A);
         expand_i8_raw(v1, mrow, c0, cols, Bv);
 #pragma unroll
         for (int q = 0; q < 8; ++q) decompose_word(N, A[q], Bv[q], A[q], Bv[q]);
-        store_unit_top(t.hi + blk * 2048 * N.h, ru, N.h, A);
-        store_unit_top(t.lo + blk * 2048 * N.lb, ru, N.lb, Bv);
+        store_unit_top(hi, ru, N.h, A);
+        store_unit_top(lo, ru, N.lb, Bv);
     } else if (OP == OP_RECOMPOSE) {
-        load_packed_raw(t.hi + blk * 2048 * N.h, ru, N.h, p0);
-        load_packed_raw(t.lo + blk * 2048 * N.lb, ru, N.lb, p1);
+        load_packed_raw(hi, ru, N.h, p0);
+        load_packed_raw(lo, ru, N.lb, p1);
         expand_packed_raw(p0, N.h, A);
         expand_packed_raw(p1, N.lb, Bv);
 #pragma unroll
@@ -363,14 +347,14 @@ __device__ __forceinline__ void do_unit(const TensorView& t, int64_t unit_index,
         store_unit_i8(wrow, c0, t.cols, vec_ok, A);
     } else if (OP == OP_DROP_LOW) {
         load_i8_raw(wrow, c0, cols, vec_ok, v0);
-        load_packed_raw(t.lo + blk * 2048 * N.lb, ru, N.lb, p1);
+        load_packed_raw(lo, ru, N.lb, p1);
         expand_i8_raw(v0, wrow, c0, cols, A);
         expand_packed_raw(p1, N.lb, Bv);
 #pragma unroll
         for (int q = 0; q < 8; ++q) A[q] = row_in ? drop_low_word(N, A[q], Bv[q]) : 0u;
-        store_unit_top(t.hi + blk * 2048 * N.h, ru, N.h, A);
+        store_unit_top(hi, ru, N.h, A);
     } else if (OP == OP_UNPACK) {
-        load_packed_raw(t.hi + blk * 2048 * bits, ru, bits, p0);
+        load_packed_raw(hi, ru, bits, p0);
         expand_packed_raw(p0, bits, A);
 #pragma unroll
         for (int q = 0; q < 8; ++q) A[q] = top_to_values(A[q], bits);
@@ -380,8 +364,72 @@ __device__ __forceinline__ void do_unit(const TensorView& t, int64_t unit_index,
         expand_i8_raw(v0, wrow, c0, cols, A);
 #pragma unroll
         for (int q = 0; q < 8; ++q) A[q] = values_to_top(A[q], bits);
-        store_unit_top(t.hi + blk * 2048 * bits, ru, bits, A);
+        store_unit_top(hi, ru, bits, A);
     }
+}
+
+// A thread's share of the work is a PAIR of units 64 rows apart in the same 128 x 128 block, so that one index
+// decode and one set of base pointers serves both (these kernels are bound by integer instructions, not by
+// bandwidth).  pair_index walks the tensor in this order, fastest first: the 32 lanes of a warp (four units of each
+// of eight consecutive rows of one block), the column groups, the eight 8-row bands of the block's upper half, the
+// row blocks.  Consecutive warps read or write consecutive 128-byte lines of the same int8 rows; every packed access
+// of a warp is one contiguous run of 512 / 256 / 128 bytes.  All index arithmetic is 32-bit (the entry points refuse
+// tensors of 2^31 rows, columns or blocks); only the final byte offsets are widened.
+template <int OP, class NestT>
+__device__ __forceinline__ void do_pair(const TensorView& t, uint32_t pair_index, const NestT& N, int bits) {
+    const uint32_t groups = (uint32_t)((t.cols + 127) >> 7);
+    const uint32_t wi = pair_index >> 5, x = pair_index & 31u;
+    const uint32_t band = wi / groups, g = wi - band * groups;
+    const uint32_t rb = band >> 3, r8 = band & 7u;
+    const uint32_t blk = rb * groups + g;
+    const int ru = (int)(r8 * 32u + x);                       // row-in-block * 4 + unit of the first unit of the pair
+    const uint32_t row = rb * 128u + (uint32_t)(ru >> 2);
+    const uint32_t c0 = (g * 4u + (x & 3u)) * 32u;
+    const int hbits = (OP == OP_UNPACK || OP == OP_PACK) ? bits : N.h;
+    uint8_t* hi = t.hi + (uint64_t)blk * (uint32_t)(2048 * hbits);
+    uint8_t* lo = (OP == OP_UNPACK || OP == OP_PACK) ? nullptr : t.lo + (uint64_t)blk * (uint32_t)(2048 * N.lb);
+    const bool vec_ok = ((t.ld & 15) == 0) && ((reinterpret_cast<uintptr_t>(t.w) & 15) == 0) &&
+                        (OP != OP_DECOMPOSE || (reinterpret_cast<uintptr_t>(t.mask) & 15) == 0);
+    const uint32_t ld = (uint32_t)t.ld, rows = (uint32_t)t.rows;
+    int8_t* wrow = t.w + (uint64_t)row * ld;
+    const int8_t* mrow = OP == OP_DECOMPOSE ? reinterpret_cast<const int8_t*>(t.mask) + (uint64_t)row * ld : nullptr;
+    if (OP == OP_RECOMPOSE || OP == OP_UNPACK) {
+        // packed -> int8 moves few bytes per thread: both units' loads are issued before either is expanded
+        const int fb = OP == OP_UNPACK ? bits : N.h;
+        PackedRaw a0, a1, b0, b1;
+        const bool in0 = row < rows, in1 = row + 64u < rows;
+        if (in0) { load_packed_raw(hi, ru, fb, a0); if (OP == OP_RECOMPOSE) load_packed_raw(lo, ru, N.lb, a1); }
+        if (in1) { load_packed_raw(hi, ru + 256, fb, b0); if (OP == OP_RECOMPOSE) load_packed_raw(lo, ru + 256, N.lb, b1); }
+        uint32_t A[8], Bv[8];
+        if (in0) {
+            expand_packed_raw(a0, fb, A);
+            if (OP == OP_RECOMPOSE) {
+                expand_packed_raw(a1, N.lb, Bv);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) A[q] = recompose_word(N, A[q], Bv[q]);
+            } else {
+#pragma unroll
+                for (int q = 0; q < 8; ++q) A[q] = top_to_values(A[q], bits);
+            }
+            store_unit_i8(wrow, c0, t.cols, vec_ok, A);
+        }
+        if (in1) {
+            expand_packed_raw(b0, fb, A);
+            if (OP == OP_RECOMPOSE) {
+                expand_packed_raw(b1, N.lb, Bv);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) A[q] = recompose_word(N, A[q], Bv[q]);
+            } else {
+#pragma unroll
+                for (int q = 0; q < 8; ++q) A[q] = top_to_values(A[q], bits);
+            }
+            store_unit_i8(wrow + (uint64_t)64 * ld, c0, t.cols, vec_ok, A);
+        }
+        return;
+    }
+    unit_body<OP>(t, N, bits, hi, lo, ru, wrow, mrow, c0, row < rows, vec_ok);
+    unit_body<OP>(t, N, bits, hi, lo, ru + 256, wrow + (uint64_t)64 * ld, OP == OP_DECOMPOSE ? mrow + (uint64_t)64 * ld : nullptr, c0,
+                  row + 64u < rows, vec_ok);
 }
 
 template <int OP, class NestT>
@@ -389,7 +437,7 @@ __global__ void __launch_bounds__(256, 4) codec_kernel(TensorView t, int64_t tot
     const NestT N(n, h, comp);
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < total_units; u += stride)
-        do_unit<OP>(t, u, N, bits);
+        do_pair<OP>(t, (uint32_t)u, N, bits);
 }
 
 // one launch over a whole model: table entries carry the running unit count
@@ -403,9 +451,10 @@ struct BatchEntry {
 };
 static_assert(sizeof(BatchEntry) == 64, "table entry is 64 bytes");
 
-// A model is cut into work items of one 128 x 128 block (512 units) each, none of which straddles two tensors;
-// block b of the batched launch takes items b, b + grid, ..., so no thread ever searches the tensor table.
-constexpr int kItemUnits = 512;
+// A model is cut into work items of 256 consecutive unit pairs (a tensor's pair count is a multiple of 256, so no
+// item straddles two tensors); block b of the batched launch takes items b, b + grid, ..., so no thread ever
+// searches the tensor table.
+constexpr int kItemUnits = 256;      // unit pairs per work item: one per thread of a block, one 128 x 128 block of a tensor
 constexpr int kBatchBlocksPerSM = 4;
 struct BatchItem {
     int32_t entry;          // which tensor
@@ -425,7 +474,7 @@ __global__ void __launch_bounds__(256, 4) codec_batched_kernel(const BatchEntry*
         TensorView t;
         t.rows = __ldg(&e->rows); t.cols = __ldg(&e->cols); t.ld = __ldg(&e->ld);
         t.hi = e->hi; t.lo = e->lo; t.w = e->w; t.mask = nullptr;
-        for (int i = threadIdx.x; i < item.units; i += blockDim.x) do_unit<OP>(t, item.first_unit + i, N, 0);
+        for (int i = threadIdx.x; i < item.units; i += blockDim.x) do_pair<OP>(t, (uint32_t)(item.first_unit + i), N, 0);
     }
 }
 
@@ -470,6 +519,15 @@ __global__ void __launch_bounds__(256) word64_to_sliced_kernel(const uint64_t* _
         }
         store_unit_top(packed + ((row >> 7) * groups + (ur >> 2)) * 2048 * BITS, (int)((row & 127) * 4 + (ur & 3)), BITS, T);
     }
+}
+
+// unit pairs (the work of one thread, see do_pair) of a [rows, cols] tensor: 256 per 128 x 128 block
+inline int64_t walk_units(int64_t rows, int64_t cols) {
+    return ((rows + 127) / 128) * ((cols + 127) / 128) * 256;
+}
+// the 32-bit index arithmetic of the kernels covers tensors below 2^31 rows, row pitch and pairs
+inline bool walk_fits(int64_t rows, int64_t cols, int64_t ld) {
+    return rows < (1ll << 31) - 128 && cols < (1ll << 31) - 128 && ld < (1ll << 31) && walk_units(rows, cols) < (1ll << 31);
 }
 
 inline int launch_blocks(int64_t total_units) {
@@ -530,7 +588,8 @@ void dispatch_nest(bool batched, const TensorView& t, const BatchEntry* table, i
 template <int OP>
 int run_single(TensorView t, int n, int h, int comp, int bits, void* stream) {
     if (t.rows == 0 || t.cols == 0) return NQ_OK;
-    int64_t total = ((t.rows + 127) / 128) * ((t.cols + 127) / 128) * 512;       // whole blocks, 512 units each
+    if (!walk_fits(t.rows, t.cols, t.ld)) return NQ_ERR_UNSUPPORTED;
+    int64_t total = walk_units(t.rows, t.cols);
     if (OP == OP_UNPACK || OP == OP_PACK) launch_one<OP, Nest>(t, total, n, h, comp, bits, (cudaStream_t)stream);
     else dispatch_nest<OP>(false, t, nullptr, 0, total, n, h, comp, (cudaStream_t)stream);
     return cudaGetLastError() == cudaSuccess ? NQ_OK : NQ_ERR_CUDA;
@@ -628,7 +687,7 @@ int nq_pack(const int8_t* values, int64_t ld, int bits, int64_t rows, int64_t co
 }
 
 static int64_t items_of(const nq_tensor_desc& d) {
-    return ((d.rows + 127) / 128) * ((d.cols + 127) / 128);              // one item per 128 x 128 block
+    return walk_units(d.rows, d.cols) / kItemUnits;
 }
 
 int64_t nq_batch_table_bytes(const nq_tensor_desc* descs, int count) {
@@ -655,6 +714,7 @@ int nq_batch_plan(const nq_tensor_desc* descs, int count, void* table, int64_t t
     for (int i = 0; i < count; ++i) {
         const nq_tensor_desc& d = descs[i];
         if (d.ld < d.cols) return NQ_ERR_INVALID_ARG;
+        if (!walk_fits(d.rows, d.cols, d.ld)) return NQ_ERR_UNSUPPORTED;
         if (d.rows > 0 && d.cols > 0) {
             if (!d.packed_high || !d.packed_low || !d.w_int) return NQ_ERR_INVALID_ARG;
             if (!aligned16(d.packed_high) || !aligned16(d.packed_low) || !aligned16(d.w_int) || (d.ld & 15))
@@ -664,7 +724,7 @@ int nq_batch_plan(const nq_tensor_desc* descs, int count, void* table, int64_t t
         e.rows = d.rows; e.cols = d.cols; e.ld = d.ld;
         e.hi = (uint8_t*)d.packed_high; e.lo = (uint8_t*)d.packed_low; e.w = d.w_int;
         e.first_unit = units_before; e.pad_ = 0;
-        const int64_t units = items_of(d) * kItemUnits;
+        const int64_t units = walk_units(d.rows, d.cols);
         units_before += units;
         for (int64_t u = 0; u < units; u += kItemUnits) {
             BatchItem& it = items[n_items++];

@@ -251,8 +251,11 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
         // as deep a ring of packed tiles as shared memory allows: it is what hides the load latency of B
         // (pair kernel: a multiple of its unpack group count, see nq_contraction_pair.cuh)
         a.packed_stages = 0;
-        // pair kernel, part-bit: every width is read straight from the packed tensor's blocks (contiguous, coalesced)
-        direct = !nest && pair && direct_fetch_enabled();
+        // pair kernel, part-bit: fields of 1, 2 and 4 bits are read straight from the packed tensor's blocks (one
+        // coalesced load per 32 fields); wider fields come through the ring, whose slots are filled by one bulk copy
+        // per block (measured, 16384^3: direct reads of h = 5 / 6 / 7 need two or three loads per unit in flight for
+        // four stages and fall to 2.3 / 2.3 / 1.75 POP/s against 2.97 / 2.64 / 2.35 through the ring)
+        direct = !nest && pair && (h_bits == 1 || h_bits == 2 || h_bits == 4) && direct_fetch_enabled();
         const bool high_in_ring = !nest || h_bits > l + 1;
         const int ring_bits = high_in_ring ? h_bits : l + 1;
         const int direct_bits = nest ? (high_in_ring ? l + 1 : h_bits) : h_bits;
