@@ -217,6 +217,17 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
             if (cost < best) { best = cost; bn = cand_bn[c]; pair = cand_pair[c]; }
         }
     }
+    // Full-bit with short K: a CTA's epilogue warps need a time that does not depend on K for their 128 x 256
+    // outputs (about 6500 cycles; 7800 when the accumulator hand-back crosses a CTA pair), so once the MMAs of a tile
+    // take less than that the tile is epilogue-bound and single CTAs are faster (measured at M = 50432, K = 768:
+    // N = 2304 122 -> 102 us, N = 3072 150 -> 135 us; K = 3072 stays on pairs, 90 against 126 us).
+    if (pair && !part && N > 128 && k_blocks * 560.0 < 7800.0) {
+        const long long nt = (N + 255) / 256;
+        const double waves_pair = (double)((((m_tiles + 1) / 2) * nt + sms / 2 - 1) / (sms / 2));
+        const double waves_single = (double)(((long long)m_tiles * nt + sms - 1) / sms);
+        const double mma_single = k_blocks * 800.0;
+        if (waves_single * (mma_single > 6500.0 ? mma_single : 6500.0) < waves_pair * 7800.0) { pair = false; bn = 256; }
+    }
     const int b_box_rows = pair ? kPairBN / 2 : bn;
     ContractionArgs a{};
     if (geom) a.g = *geom;
