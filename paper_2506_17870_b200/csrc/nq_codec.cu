@@ -440,41 +440,53 @@ __global__ void __launch_bounds__(256, 4) codec_kernel(TensorView t, int64_t tot
         do_pair<OP>(t, (uint32_t)u, N, bits);
 }
 
-// one launch over a whole model: table entries carry the running unit count
-struct BatchEntry {
-    int64_t rows, cols, ld;
+// One launch over a whole model.  The model is cut into work items of 256 consecutive unit pairs -- one 128 x 128
+// block of one tensor, one pair per thread of a block -- and every item carries all a block needs (base pointers,
+// shape, pitch, first pair), so that a thread block reads ONE 48-byte descriptor per item, with no second look-up
+// behind it.  Block b takes items b, b + grid, ...; the next item's descriptor is fetched before the current item
+// is worked on.  (The first version read an item, then the tensor's table entry, then the data: three dependent
+// trips to memory per item, a third of the time of a ResNet-101-sized switch.)
+constexpr int kItemUnits = 256;      // unit pairs per work item
+constexpr int kBatchBlocksPerSM = 4;
+struct BatchItem {
     uint8_t* hi;
     uint8_t* lo;
     int8_t* w;
-    int64_t first_unit;     // units of all earlier tensors
-    int64_t pad_;
+    int32_t rows, cols, ld;
+    uint32_t first_pair;    // first pair of the item inside its tensor
+    uint32_t pad_[2];
 };
-static_assert(sizeof(BatchEntry) == 64, "table entry is 64 bytes");
+static_assert(sizeof(BatchItem) == 48, "work item is three 16-byte words");
 
-// A model is cut into work items of 256 consecutive unit pairs (a tensor's pair count is a multiple of 256, so no
-// item straddles two tensors); block b of the batched launch takes items b, b + grid, ..., so no thread ever
-// searches the tensor table.
-constexpr int kItemUnits = 256;      // unit pairs per work item: one per thread of a block, one 128 x 128 block of a tensor
-constexpr int kBatchBlocksPerSM = 4;
-struct BatchItem {
-    int32_t entry;          // which tensor
-    int32_t units;          // how many units of it (<= kItemUnits)
-    int64_t first_unit;     // first unit inside that tensor
-};
-static_assert(sizeof(BatchItem) == 16, "work item is 16 bytes");
+__device__ __forceinline__ BatchItem load_item(const BatchItem* items, int b) {
+    const uint4* p = reinterpret_cast<const uint4*>(items + b);
+    const uint4 a = __ldg(p), c = __ldg(p + 1), d = __ldg(p + 2);
+    BatchItem it;
+    it.hi = reinterpret_cast<uint8_t*>(((uint64_t)a.y << 32) | a.x);
+    it.lo = reinterpret_cast<uint8_t*>(((uint64_t)a.w << 32) | a.z);
+    it.w = reinterpret_cast<int8_t*>(((uint64_t)c.y << 32) | c.x);
+    it.rows = (int32_t)c.z; it.cols = (int32_t)c.w; it.ld = (int32_t)d.x; it.first_pair = d.y;
+    return it;
+}
 
 template <int OP, class NestT>
-__global__ void __launch_bounds__(256, 4) codec_batched_kernel(const BatchEntry* __restrict__ table,
-                                                               const BatchItem* __restrict__ items, int n_items,
+__global__ void __launch_bounds__(256, 4) codec_batched_kernel(const BatchItem* __restrict__ items, int n_items,
                                                                int n, int h, int comp) {
     const NestT N(n, h, comp);
-    for (int b = blockIdx.x; b < n_items; b += gridDim.x) {
-        const BatchItem item = items[b];
-        const BatchEntry* e = table + item.entry;
+    int b = blockIdx.x;
+    if (b >= n_items) return;
+    BatchItem cur = load_item(items, b);
+    while (true) {
+        const int nb = b + (int)gridDim.x;
+        BatchItem nxt = cur;
+        if (nb < n_items) nxt = load_item(items, nb);          // in flight while this item is worked on
         TensorView t;
-        t.rows = __ldg(&e->rows); t.cols = __ldg(&e->cols); t.ld = __ldg(&e->ld);
-        t.hi = e->hi; t.lo = e->lo; t.w = e->w; t.mask = nullptr;
-        for (int i = threadIdx.x; i < item.units; i += blockDim.x) do_pair<OP>(t, (uint32_t)(item.first_unit + i), N, 0);
+        t.rows = cur.rows; t.cols = cur.cols; t.ld = cur.ld;
+        t.hi = cur.hi; t.lo = cur.lo; t.w = cur.w; t.mask = nullptr;
+        do_pair<OP>(t, cur.first_pair + threadIdx.x, N, 0);
+        if (nb >= n_items) break;
+        cur = nxt;
+        b = nb;
     }
 }
 
@@ -545,30 +557,28 @@ void launch_one(const TensorView& t, int64_t total, int n, int h, int comp, int 
     codec_kernel<OP, NestT><<<launch_blocks(total), 256, 0, s>>>(t, total, n, h, comp, bits);
 }
 template <int OP, class NestT>
-void launch_batch(const BatchEntry* table, int count, int64_t items, int n, int h, int comp, cudaStream_t s) {
-    const BatchItem* list = reinterpret_cast<const BatchItem*>(table + count);
+void launch_batch(const BatchItem* list, int64_t items, int n, int h, int comp, cudaStream_t s) {
     // as many blocks as are resident at once (four per SM); a block walks the items b, b + grid, ...: with small
-    // items the last round is a small part of the whole, where one block per item of 1024 units left the
-    // ResNet-101-shaped model with 2.3 rounds of blocks
+    // items the last round is a small part of the whole
     const int64_t resident = (int64_t)nq::sm_count() * kBatchBlocksPerSM;
     const unsigned grid = (unsigned)(items < resident ? items : resident);
-    codec_batched_kernel<OP, NestT><<<grid, 256, 0, s>>>(table, list, (int)items, n, h, comp);
+    codec_batched_kernel<OP, NestT><<<grid, 256, 0, s>>>(list, (int)items, n, h, comp);
 }
 
 template <int OP, int H>
-void dispatch_comp(bool batched, const TensorView& t, const BatchEntry* table, int count, int64_t total, int comp,
+void dispatch_comp(bool batched, const TensorView& t, const BatchItem* table, int count, int64_t total, int comp,
                    cudaStream_t s) {
     if (comp) {
-        if (batched) launch_batch<OP, SNest<8, H, 1>>(table, count, total, 8, H, 1, s);
+        if (batched) launch_batch<OP, SNest<8, H, 1>>(table, total, 8, H, 1, s);
         else launch_one<OP, SNest<8, H, 1>>(t, total, 8, H, 1, 0, s);
     } else {
-        if (batched) launch_batch<OP, SNest<8, H, 0>>(table, count, total, 8, H, 0, s);
+        if (batched) launch_batch<OP, SNest<8, H, 0>>(table, total, 8, H, 0, s);
         else launch_one<OP, SNest<8, H, 0>>(t, total, 8, H, 0, 0, s);
     }
 }
 
 template <int OP>
-void dispatch_nest(bool batched, const TensorView& t, const BatchEntry* table, int count, int64_t total, int n, int h,
+void dispatch_nest(bool batched, const TensorView& t, const BatchItem* table, int count, int64_t total, int n, int h,
                    int comp, cudaStream_t s) {
     if (n == 8) {
         switch (h) {
@@ -581,7 +591,7 @@ void dispatch_nest(bool batched, const TensorView& t, const BatchEntry* table, i
             default: return dispatch_comp<OP, 7>(batched, t, table, count, total, comp, s);
         }
     }
-    if (batched) launch_batch<OP, Nest>(table, count, total, n, h, comp, s);
+    if (batched) launch_batch<OP, Nest>(table, total, n, h, comp, s);
     else launch_one<OP, Nest>(t, total, n, h, comp, 0, s);
 }
 
@@ -697,7 +707,7 @@ int64_t nq_batch_table_bytes(const nq_tensor_desc* descs, int count) {
         if (descs[i].rows < 0 || descs[i].cols < 0) return -1;
         items += items_of(descs[i]);
     }
-    return (int64_t)(count > 0 ? count : 1) * (int64_t)sizeof(BatchEntry) + (items > 0 ? items : 1) * (int64_t)sizeof(BatchItem);
+    return (items > 0 ? items : 1) * (int64_t)sizeof(BatchItem);
 }
 
 int nq_batch_plan(const nq_tensor_desc* descs, int count, void* table, int64_t table_bytes,
@@ -707,10 +717,8 @@ int nq_batch_plan(const nq_tensor_desc* descs, int count, void* table, int64_t t
     if (need < 0) return NQ_ERR_INVALID_ARG;
     if (table_bytes < need) return NQ_ERR_WORKSPACE;
     if (!aligned16(table)) return NQ_ERR_ALIGNMENT;
-    std::vector<unsigned char> host((size_t)need, 0);
-    BatchEntry* entries = reinterpret_cast<BatchEntry*>(host.data());
-    BatchItem* items = reinterpret_cast<BatchItem*>(host.data() + (size_t)count * sizeof(BatchEntry));
-    int64_t n_items = 0, units_before = 0;
+    std::vector<BatchItem> host((size_t)(need / (int64_t)sizeof(BatchItem)));
+    int64_t n_items = 0;
     for (int i = 0; i < count; ++i) {
         const nq_tensor_desc& d = descs[i];
         if (d.ld < d.cols) return NQ_ERR_INVALID_ARG;
@@ -720,24 +728,19 @@ int nq_batch_plan(const nq_tensor_desc* descs, int count, void* table, int64_t t
             if (!aligned16(d.packed_high) || !aligned16(d.packed_low) || !aligned16(d.w_int) || (d.ld & 15))
                 return NQ_ERR_ALIGNMENT;
         }
-        BatchEntry& e = entries[i];
-        e.rows = d.rows; e.cols = d.cols; e.ld = d.ld;
-        e.hi = (uint8_t*)d.packed_high; e.lo = (uint8_t*)d.packed_low; e.w = d.w_int;
-        e.first_unit = units_before; e.pad_ = 0;
-        const int64_t units = walk_units(d.rows, d.cols);
-        units_before += units;
-        for (int64_t u = 0; u < units; u += kItemUnits) {
-            BatchItem& it = items[n_items++];
-            it.entry = i;
-            it.units = (int32_t)((units - u) < kItemUnits ? (units - u) : kItemUnits);
-            it.first_unit = u;
+        const int64_t pairs = (d.rows > 0 && d.cols > 0) ? walk_units(d.rows, d.cols) : 0;
+        for (int64_t u = 0; u < pairs; u += kItemUnits) {
+            BatchItem& it = host[(size_t)n_items++];
+            it.hi = (uint8_t*)d.packed_high; it.lo = (uint8_t*)d.packed_low; it.w = d.w_int;
+            it.rows = (int32_t)d.rows; it.cols = (int32_t)d.cols; it.ld = (int32_t)d.ld;
+            it.first_pair = (uint32_t)u; it.pad_[0] = it.pad_[1] = 0;
         }
     }
     *work_items_out = n_items;
     if (count == 0 || n_items == 0) return NQ_OK;
     // the source is pageable host memory: the runtime stages it before this call returns
-    cudaError_t err = cudaMemcpyAsync(table, host.data(), (size_t)count * sizeof(BatchEntry) + (size_t)n_items * sizeof(BatchItem),
-                                      cudaMemcpyHostToDevice, (cudaStream_t)stream);
+    cudaError_t err = cudaMemcpyAsync(table, host.data(), (size_t)n_items * sizeof(BatchItem), cudaMemcpyHostToDevice,
+                                      (cudaStream_t)stream);
     return err == cudaSuccess ? NQ_OK : NQ_ERR_CUDA;
 }
 
@@ -745,7 +748,7 @@ static int run_batched(int op, const void* table, int count, int64_t units, int 
     if (count < 0 || units < 0 || units > 0x7fffffffLL || !table) return NQ_ERR_INVALID_ARG;
     if (!nest_ok(n, h)) return NQ_ERR_UNSUPPORTED;
     if (count == 0 || units == 0) return NQ_OK;
-    const BatchEntry* entries = reinterpret_cast<const BatchEntry*>(table);
+    const BatchItem* entries = reinterpret_cast<const BatchItem*>(table);
     TensorView none{};
     if (op == OP_RECOMPOSE) dispatch_nest<OP_RECOMPOSE>(true, none, entries, count, units, n, h, comp, (cudaStream_t)stream);
     else dispatch_nest<OP_DROP_LOW>(true, none, entries, count, units, n, h, comp, (cudaStream_t)stream);
