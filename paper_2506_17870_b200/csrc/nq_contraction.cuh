@@ -33,7 +33,7 @@ __host__ __device__ constexpr int stages_for(int bn, bool part) {
     return part ? (bn == 64 ? 6 : bn == 128 ? 4 : 3) : (bn == 64 ? 8 : bn == 128 ? 6 : 4);
 }
 constexpr int kMaxPackedStages = 8;     // ring of packed (still INTh) B tiles; the depth in use is chosen by the host
-constexpr int kGroupM = 16;        // tile rasterisation: 16 M-tiles share a band of N-tiles
+constexpr int kGroupM = 16;        // tile rasterisation: at most 16 M-tiles share a band of N-tiles (the host picks 4, 8 or 16)
 
 // How the A operand is gathered.
 //   kModeGemm    A is a plain [M, K] matrix: one 2-D tile per stage.
@@ -68,7 +68,8 @@ struct ContractionArgs {
     ConvGeom g;
     int M, N, K;
     int m_tiles, n_tiles, k_blocks;
-    FastDiv div_group, div_last;   // by kGroupM * n_tiles, and by the row count of the last (short) group of M-tiles
+    int group_log2;                // M-tiles per rasterisation group = 2^group_log2
+    FastDiv div_group, div_last;   // by (group size) * n_tiles, and by the row count of the last (short) group of M-tiles
     const float* w_scale;
     const float* bias;
     float act_scale;
@@ -132,13 +133,14 @@ __host__ __device__ inline int contraction_smem_bytes(int bn, bool part, int h_b
 }
 
 __device__ __forceinline__ void tile_coords(int tile, const ContractionArgs& p, int& mt, int& nt) {
-    const int per_group = kGroupM * p.n_tiles;
+    const int gm = 1 << p.group_log2;
+    const int per_group = gm * p.n_tiles;
     const int g = (int)fast_div((uint32_t)tile, p.div_group);
-    const int first = g * kGroupM;
+    const int first = g * gm;
     const int local = tile - g * per_group;
-    if (p.m_tiles - first >= kGroupM) {                  // a full group: kGroupM is a power of two
-        mt = first + (local & (kGroupM - 1));
-        nt = local / kGroupM;
+    if (p.m_tiles - first >= gm) {                       // a full group: its size is a power of two
+        mt = first + (local & (gm - 1));
+        nt = local >> p.group_log2;
     } else {
         const int gsz = p.m_tiles - first;
         nt = (int)fast_div((uint32_t)local, p.div_last);

@@ -235,8 +235,18 @@ int run_contraction(const CUtensorMap& tmA, int mode, const ConvGeom* geom, int 
     a.m_tiles = pair ? (m_tiles + 1) / 2 : m_tiles;
     a.n_tiles = (int)((N + bn - 1) / bn);
     a.k_blocks = k_blocks;
-    a.div_group = make_fastdiv((uint32_t)(kGroupM * a.n_tiles));
-    a.div_last = make_fastdiv((uint32_t)((a.m_tiles % kGroupM) ? (a.m_tiles % kGroupM) : 1));
+    // Rasterisation: a group of M-tiles shares a band of N-tiles, so that the group's rows of A stay in L2 while the
+    // N-tiles go by.  The band must fit beside the stream of B and the output: about 32 MB of A rows per group
+    // (16 M-tiles up to K = 8192 on pairs; 8 at K = 16384, where 16 made every wave re-read its 67 MB band: measured
+    // 5.2-7.0 GB of DRAM traffic per 16384^3 launch against 1.07 GB algorithmic).
+    {
+        const double band_rows = (pair ? 256.0 : 128.0) * kGroupM;
+        int gl = 4;
+        while (gl > 2 && band_rows / kGroupM * (1 << gl) * (double)K > 34.0e6) --gl;
+        a.group_log2 = gl;
+    }
+    a.div_group = make_fastdiv((uint32_t)((1 << a.group_log2) * a.n_tiles));
+    a.div_last = make_fastdiv((uint32_t)((a.m_tiles % (1 << a.group_log2)) ? (a.m_tiles % (1 << a.group_log2)) : 1));
     a.w_scale = w_scale; a.bias = bias; a.act_scale = act_scale;
     a.acc_out = acc_out; a.ld_acc = ld_acc; a.y = Y; a.ldy = ldy; a.y_is_bf16 = (y_dtype == NQ_BF16);
     a.y_is_i8 = (y_dtype == kOutI8 && oq) ? 1 : 0;
