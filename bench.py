@@ -1090,7 +1090,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--sizes", default=",".join(map(str, SIZES)))
-    ap.add_argument("--cpu-rows", type=int, default=256)
+    ap.add_argument("--cpu-rows", type=int, default=4096)
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--conv-batch", type=int, default=32)
     ap.add_argument("--no-conv", dest="conv", action="store_false")

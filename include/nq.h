@@ -337,6 +337,9 @@ NQ_API int nq_avgpool_requant_nhwc_i8(const int8_t *X, int B, int H, int W, int 
  *     overwrite every byte they later read, so nothing has to be cleared between calls; but two calls
  *     whose work overlaps on the GPU (different streams, or different host threads) would scribble over
  *     each other's staging data.  Keep calls on one stream, or order them yourself.
+ *   - Host side: the looked-up address is cached per device (devices 0..63) in the library; host threads may
+ *     make their calls in any order, the first one included.  A cached address does not survive
+ *     cudaDeviceReset: a process that resets a device must not call this function on it afterwards.
  *   - No cudaMalloc, cudaFree or allocating library routine is called.
  * Arguments, layouts, results and error codes are otherwise those of nq_conv_implicit_gemm.
  */

@@ -5,8 +5,9 @@
 // and, per slice of width s, s words on the packed side.  Units are walked block by block (128 rows x 128
 // columns, the packed layout's storage unit), rows fastest: the 32 lanes of a warp hold four units of each of
 // eight consecutive rows, so every packed access of a warp is one contiguous run (512 / 256 / 128 bytes of the
-// 4- / 2- / 1-bit slice) and every int8 access covers eight whole 128-byte lines.  One thread owns one unit at a time and
-// keeps it in registers as eight "top-aligned" words T[q]: byte lane i of T[q] holds the k-bit
+// 4- / 2- / 1-bit slice) and every int8 access covers eight whole 128-byte lines.  One thread takes a PAIR of units
+// per loop trip -- the same columns, 64 rows apart in the block, so one index decode serves both and the loads of
+// both are in flight together -- and keeps each in registers as eight "top-aligned" words T[q]: byte lane i of T[q] holds the k-bit
 // field of element 4q+i in its TOP k bits.  In that form every slice is a fixed bit range of every
 // byte, so moving between T and the slices is a mask, a shift and an OR per word -- four elements
 // per instruction -- and the nesting arithmetic (Eq. 5, 6, 10) is done on four bytes at a time.

@@ -9,6 +9,8 @@
 //     workspace and the plain GEMM path runs on it.
 #include <cuda.h>
 #include <cuda_runtime.h>
+
+#include <atomic>
 #include <stdint.h>
 
 #include "../../include/nq.h"
@@ -358,15 +360,16 @@ int nq_conv_implicit_gemm_static(const int8_t* X, const void* Wt, int64_t ldw, i
     if (need < 0) return NQ_ERR_INVALID_ARG;
     if (need > (int64_t)NQ_CONV_STATIC_SCRATCH_BYTES) return NQ_ERR_WORKSPACE;   // does not fit the built-in staging array
     // device address of the array, looked up once per device with that device current
-    static unsigned char* base[64] = {nullptr};
+    // (atomic slots: two host threads that both make a device's first call store the same address)
+    static std::atomic<unsigned char*> base[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return NQ_ERR_CUDA;
-    if (!base[dev]) {
-        unsigned char* ptr = nullptr;
+    unsigned char* ptr = base[dev].load(std::memory_order_relaxed);
+    if (!ptr) {
         if (cudaGetSymbolAddress((void**)&ptr, g_conv_static_scratch) != cudaSuccess || !ptr) return NQ_ERR_CUDA;
-        base[dev] = ptr;
+        base[dev].store(ptr, std::memory_order_relaxed);
     }
-    unsigned char* ws = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(base[dev]) + 1023) & ~uintptr_t(1023));
+    unsigned char* ws = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(ptr) + 1023) & ~uintptr_t(1023));
     return nq_conv_implicit_gemm(X, Wt, ldw, part_bit, n_bits, h_bits, d, w_scale, act_scale, bias, acc_out, Y, y_dtype,
                                  ws, NQ_CONV_STATIC_SCRATCH_BYTES, stream);
 }

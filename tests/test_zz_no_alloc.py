@@ -5,13 +5,15 @@ that only ever sees the buffers its host application hands it, a control loop th
 allocator).  nq_conv_implicit_gemm_static serves them: same inputs and outputs, no workspace, staging
 through an array built into the library.  This file checks, through the C boundary, that it returns
 exactly what nq_conv_implicit_gemm returns -- bit-exact INT32 accumulators and identical fp32 outputs,
-the bar the other convolution tests use -- on two calls in a row that reuse the shared array, and that a
-layer too large for the array is refused.  It is named so that pytest collects it after every other test.
+the bar the other convolution tests use -- on two calls in a row that reuse the shared array, that its result is
+the CPU oracle's direct convolution, that the device's free memory is the same before and after a call, and that
+a layer too large for the array is refused.  It is named so that pytest collects it after every other test.
 """
 import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2506_17870_b200 as nq
 from paper_2506_17870_b200 import workloads as wl
 
@@ -52,6 +54,32 @@ def test_two_calls_in_a_row_match_the_ordinary_entry_point():
     _compare(big, 8, 1, part=False)
     _compare(small, 2, 2, part=True)
     _compare(big, 8, 3, part=True)
+
+
+def test_result_is_the_oracles_convolution_and_no_device_memory_is_taken():
+    """Full-bit and part-bit (Eq. 9) results of the allocation-free call against the oracle's direct convolution
+    (accumulators bit-exact, fp32 output equal), with the driver's free-memory figure read around the second call:
+    the first call has looked the array's address up, so the second must leave the figure where it was."""
+    L = wl.ConvLayer("c64s2", 64, 18, 18, 128, 3, 3, 2, 1)
+    batch = 3
+    d = wl.conv_layer_inputs(73, 5, L, batch)
+    wh, _ = oracle.decompose(d["W"], d["mask"], 8, 6, True)
+    desc, x, w, hi, ws, sa = _layer_tensors(L, batch, 5)
+    for part in (False, True):
+        ref = oracle.conv_acc(d["X"], wh if part else d["W"], L.stride, L.pad).transpose(0, 2, 3, 1)
+        acc = torch.full((batch, L.Ho, L.Wo, L.Cout), -1, dtype=torch.int32, device="cuda")
+        y = torch.full((batch, L.Ho, L.Wo, L.Cout), float("nan"), dtype=torch.float32, device="cuda")
+        weights = hi if part else w
+        nq.nq_conv_implicit_gemm_static(x, weights, desc, ws, sa, acc, y, part_bit=part, n_bits=8, h_bits=6)
+        torch.cuda.synchronize()
+        free_before, _ = torch.cuda.mem_get_info()
+        nq.nq_conv_implicit_gemm_static(x, weights, desc, ws, sa, acc, y, part_bit=part, n_bits=8, h_bits=6)
+        torch.cuda.synchronize()
+        free_after, _ = torch.cuda.mem_get_info()
+        nq.nq_device_status()
+        assert free_after == free_before
+        assert np.array_equal(acc.cpu().numpy(), ref)
+        assert np.array_equal(y.cpu().numpy(), oracle.dequant(ref, d["w_scale"], sa, 2 if part else 0))
 
 
 def test_layer_larger_than_the_built_in_array_is_refused():
