@@ -74,6 +74,7 @@ def write_table(csv_path: Path, sizes, out_path: Path, command: str = "") -> Non
 
 def load(path: Path):
     """({(size, h): bytes}, None), or (None, reason) when the table is absent or was taken on other kernel sources."""
+    path = Path(path)
     if not path.exists():
         return None, "no capture on record"
     table, recorded = {}, None
