@@ -50,10 +50,7 @@ constexpr int kPairStagesPart = 4;
 // on the leader's barrier across the cluster) of different stages overlap.  Ring depths are multiples of the
 // group count, so that a ring slot is always served by the same group, in order: a parity wait is only valid
 // for a waiter that is at most one phase behind.
-#ifndef NQ_UNPACK_GROUPS
-#define NQ_UNPACK_GROUPS 4
-#endif
-constexpr int kUnpackGroups = NQ_UNPACK_GROUPS;
+constexpr int kUnpackGroups = 4;
 constexpr int kUnpackGroupWarps = kUnpackWarps / kUnpackGroups;
 constexpr int kUnpackGroupThreads = kUnpackGroupWarps * 32;
 static_assert(kPairStagesPart % kUnpackGroups == 0, "a stage slot must belong to one unpack group");
